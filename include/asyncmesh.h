@@ -1,0 +1,212 @@
+/*
+ * asyncmesh.h -- C ABI of the B200 (sm_100a) AsyncMesh per-step update library.
+ *
+ * The library holds R data-parallel replicas x S pipeline stages of flat fp32
+ * parameters on ONE GPU and advances them one optimisation step per call.  A
+ * step fuses, per stage and coordinate (paper notation: m -> R, P -> S):
+ *
+ *   1. the local optimizer step of every replica          (Section 2.3, Eq. "sparta", line 1;
+ *      AdamW with decoupled weight decay, moments local)
+ *   2. the random subset S_j^t of coordinates, one per     (Section 2.3; Appendix Lemma 1:
+ *      stage and step, shared by the stage's replicas       each element independently with prob. p)
+ *   3. the snapshot of the local iterates on S_j^t, whose  (Section 3.1: the average launched at
+ *      replica average becomes usable tau steps later        step t arrives at step t + tau)
+ *   4. delayed sparse averaging on S_j^{t-tau} with the    (Section 3.1 Eq. "asparta"; Section 3.2
+ *      EMA estimate of the average staleness                 Eq. "ema" and the corrected averaging)
+ *   5. the pipeline look-ahead: last update direction      (Section 2.2)
+ *      extrapolated by the stage's delay
+ *
+ * All pointers named "device" are CUDA device pointers on the configured
+ * device; pointers named "host" are ordinary host pointers.  Every function
+ * returns 0 (ASYNCMESH_OK) or a negative code, never throws and never aborts;
+ * asyncmesh_last_error() gives the message of the calling thread's last
+ * failure.  Calls on one handle must not overlap in time.  There is no CPU
+ * fallback: without a usable CUDA device every call that needs one fails.
+ */
+#ifndef ASYNCMESH_H
+#define ASYNCMESH_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ASYNCMESH_OK 0
+#define ASYNCMESH_ERR_INVALID_ARG (-1)
+#define ASYNCMESH_ERR_OOM (-2)
+#define ASYNCMESH_ERR_CUDA (-3)
+#define ASYNCMESH_ERR_BAD_STATE (-4)
+#define ASYNCMESH_ERR_UNSUPPORTED (-5)
+#define ASYNCMESH_ERR_DEVICE_STATUS (-6)
+
+#define ASYNCMESH_MAX_REPLICAS 16u
+#define ASYNCMESH_MAX_STAGES 64u
+#define ASYNCMESH_MAX_TAU 64u
+
+/* asyncmesh_config.flags */
+#define ASYNCMESH_FLAG_SMALL_RING 1u /* diagnostic: give each compact ring slot 1/8 of
+                                        its normal capacity, so that the overflow
+                                        report (DEVICE_STATUS) can be exercised    */
+
+/* state selectors of asyncmesh_read_state */
+#define ASYNCMESH_STATE_W 0     /* weights w_i^t                               */
+#define ASYNCMESH_STATE_M 1     /* Adam first moment                           */
+#define ASYNCMESH_STATE_V 2     /* Adam second moment                          */
+#define ASYNCMESH_STATE_D 3     /* EMA staleness estimate d_i^t (Eq. "ema")    */
+#define ASYNCMESH_STATE_LOOK 4  /* look-ahead weights of the configured delay  */
+
+typedef struct asyncmesh asyncmesh;
+
+/* Device-memory callbacks.  alloc returns a device pointer aligned to at
+ * least 256 bytes, or NULL; the library calls free exactly once per pointer. */
+typedef void *(*asyncmesh_alloc_fn)(void *ctx, size_t bytes);
+typedef void (*asyncmesh_free_fn)(void *ctx, void *device_ptr);
+
+/*
+ * Problem statement (Section 2.1: P stages x m replicas; Section 2.3: subset
+ * per stage; Section 3.1: delay tau; Section 3.2: EMA coefficient lambda;
+ * Section 2.2: stage-dependent delay delta_j).  Hyper-parameters are doubles;
+ * each derived per-step scalar is formed in double and rounded to fp32 once.
+ */
+typedef struct asyncmesh_config {
+    uint32_t R;                      /* replicas, 1..ASYNCMESH_MAX_REPLICAS            */
+    uint32_t S;                      /* stages, 1..ASYNCMESH_MAX_STAGES                */
+    const uint64_t *stage_numel;     /* host [S]: parameters of stage j, 1..2^32-1     */
+    double p;                        /* subset probability, 0..1                       */
+    uint32_t tau;                    /* averaging delay in steps, 0..ASYNCMESH_MAX_TAU */
+    uint32_t flags;                  /* 0 or ASYNCMESH_FLAG_*                          */
+    double ema_beta;                 /* the paper's lambda: weight of the NEW staleness
+                                        sample in Eq. "ema"; 0 = no correction, 0..1   */
+    double lr, beta1, beta2, eps, weight_decay; /* AdamW                              */
+    uint64_t seed;                   /* Philox key of the subset rule                  */
+    const uint32_t *lookahead_delay; /* host [S] or NULL (NULL: delta_j = S - 1 - j)   */
+    int32_t device;                  /* CUDA device ordinal                            */
+    int32_t reserved;                /* must be 0                                      */
+    void *stream;                    /* cudaStream_t all work is issued on (NULL: the
+                                        legacy default stream)                         */
+    asyncmesh_alloc_fn alloc;        /* both NULL: cudaMalloc / cudaFree               */
+    asyncmesh_free_fn free;
+    void *alloc_ctx;
+} asyncmesh_config;
+
+/*
+ * Create the state: per stage W, M, V (replica-major rows [R][row_stride]),
+ * D (coordinate-major [row_stride][R]), LOOK (only where delta_j > 0) and the
+ * snapshot ring.  The library owns all of it (obtained through cfg->alloc).
+ * Moments, D and the ring start at zero, the step counter at 0, weights are
+ * unset until asyncmesh_init_params.  The config and its arrays are copied.
+ * Errors: INVALID_ARG (range checks above), OOM (allocator returned NULL: every
+ * partial allocation is released), CUDA.
+ */
+int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out);
+
+/* Release everything.  NULL is accepted and returns ASYNCMESH_OK. */
+int asyncmesh_destroy(asyncmesh *h);
+
+/*
+ * Set the initial weights w^0 of one replica of a stage (replica = -1: all
+ * replicas, the "same initialisation" of the homogeneous setup, Section 3.3).
+ * src holds n = stage_numel[stage] floats, on the device if src_on_device != 0
+ * else on the host.  Also sets w^{-1} := w^0, i.e. look-ahead = w^0.
+ * Only allowed before the first step (BAD_STATE afterwards).
+ */
+int asyncmesh_init_params(asyncmesh *h, uint32_t stage, int32_t replica,
+                          const float *src, uint64_t n, int src_on_device);
+
+/* Floats between consecutive replica rows of a stage (a multiple of 32,
+ * >= stage_numel[stage]).  Gradient buffers use the same stride. */
+int asyncmesh_row_stride(const asyncmesh *h, uint32_t stage, uint64_t *stride);
+
+/*
+ * One step t <- t + 1 of the whole mesh (items 1-5 above for every stage), in
+ * one kernel launch on the handle's stream; returns without waiting for it.
+ * grads: host array of S device pointers; grads[j] is [R][row_stride_j] fp32,
+ * 16-byte aligned, row i = gradient of replica i evaluated by the caller
+ * (Eq. "gd": at whatever delayed weights the pipeline used).  Caller-owned,
+ * read-only, and free to reuse once the stream has passed this step.
+ * ema_beta_t / lr_t < 0 keep the configured constants; values >= 0 replace them
+ * for this step only (the paper decays both over training, Section 3.3 and
+ * Appendix B.1); weight decay is applied as lr_t * weight_decay.
+ */
+int asyncmesh_step(asyncmesh *h, const float *const *grads);
+int asyncmesh_step_ex(asyncmesh *h, const float *const *grads,
+                      double ema_beta_t, double lr_t);
+
+/*
+ * The same step with gradients in HOST memory: grads_host[j] is [R][numel_j]
+ * fp32, rows contiguous (no padding).  They are copied into library-owned
+ * device staging buffers (allocated on the first call) on the handle's
+ * stream, then the step runs.  Pinned host memory makes the copies
+ * asynchronous; pageable memory works and is slower.
+ */
+int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host);
+
+/*
+ * Look-ahead weights of a stage: w^t + delay * (w^t - w^{t-1}) (Section 2.2).
+ * Returns a library-owned device pointer [R][row_stride], valid until the next
+ * step or destroy.  delay must be the stage's configured delay (the buffer the
+ * fused step wrote) or 0 (the weights themselves); anything else: UNSUPPORTED.
+ */
+int asyncmesh_lookahead_weights(asyncmesh *h, uint32_t stage, uint32_t delay,
+                                const float **out_device, uint64_t *row_stride);
+
+/*
+ * Copy out the weights of one replica (replica = -1: the replica mean, the
+ * consensus model the paper evaluates, summed in replica order and divided by
+ * R).  dst receives n = stage_numel[stage] floats, on the device if
+ * dst_on_device != 0 else on the host.  Waits for the stream; reports a pending
+ * device status (ring overflow) as DEVICE_STATUS.
+ */
+int asyncmesh_read_params(asyncmesh *h, uint32_t stage, int32_t replica,
+                          float *dst, uint64_t n, int dst_on_device);
+
+/* Copy out one replica row of any state array (ASYNCMESH_STATE_*), replica in
+ * [0, R).  Same conventions as asyncmesh_read_params. */
+int asyncmesh_read_state(asyncmesh *h, uint32_t stage, int which, int32_t replica,
+                         float *dst, uint64_t n, int dst_on_device);
+
+/*
+ * Membership of the subset S_stage^step as the device computes it: bit (mu & 7)
+ * of bitmap_host[mu >> 3] is coordinate mu; (numel + 7) / 8 bytes, host memory.
+ * Rule: Philox-4x32-10 with key = (seed lo, seed hi) and counter
+ * (mu >> 2, stage, (uint32) step, 0); coordinate mu takes word mu & 3 and is
+ * in the subset iff word < floor(p * 2^32).
+ */
+int asyncmesh_subset_mask(asyncmesh *h, uint32_t stage, uint64_t step,
+                          uint8_t *bitmap_host);
+
+/*
+ * Consensus error of a stage, sum_i ||w_i - wbar||^2 (Section 3.3), reduced on
+ * the device in double precision.  Waits for the stream.
+ */
+int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *out_host);
+
+/* Steps taken so far. */
+int asyncmesh_step_count(const asyncmesh *h, uint64_t *t);
+
+/*
+ * Bytes the last step had to move at least: per replica-coordinate 16 read
+ * (w, g, m, v) + 12 written (w, m, v), + 4 where the look-ahead is a separate
+ * buffer, + 4p for the snapshot write, + 12p once averages are being consumed
+ * (ring read, d read, d write).  Used as the numerator of the HBM roofline.
+ */
+int asyncmesh_min_bytes_last_step(const asyncmesh *h, uint64_t *bytes);
+
+/* Wait for the stream and report a device-side status word: OK, or
+ * DEVICE_STATUS if a snapshot ring slot overflowed its capacity. */
+int asyncmesh_status(asyncmesh *h);
+
+/* Run the device's Philox-4x32-10 on n (counter, key) pairs: ctr_host [n][4],
+ * key_host [n][2], out_host [n][4], all uint32 in host memory.  Test hook. */
+int asyncmesh_debug_philox(int device, const uint32_t *ctr_host,
+                           const uint32_t *key_host, uint32_t *out_host, uint64_t n);
+
+/* Message of the calling thread's most recent failure ("" if none). */
+const char *asyncmesh_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASYNCMESH_H */

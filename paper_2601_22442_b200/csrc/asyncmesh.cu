@@ -1,0 +1,757 @@
+// C ABI of the AsyncMesh step library (see include/asyncmesh.h for the contract
+// of every entry point).  Host logic only: argument checks, memory layout, the
+// per-step scalars, kernel dispatch.  All arithmetic of the method runs in the
+// kernels of step_kernel.cuh and in the small kernels below.
+#include "../../include/asyncmesh.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "step_kernel.cuh"
+
+using namespace amk;
+
+// ---------------------------------------------------------------------------
+// errors
+// ---------------------------------------------------------------------------
+
+static thread_local char g_err[512] = "";
+
+static int fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CU_TRY(expr)                                                              \
+    do {                                                                          \
+        cudaError_t e_ = (expr);                                                  \
+        if (e_ != cudaSuccess)                                                    \
+            return fail(ASYNCMESH_ERR_CUDA, "%s failed: %s", #expr,               \
+                        cudaGetErrorString(e_));                                  \
+    } while (0)
+
+extern "C" const char *asyncmesh_last_error(void) { return g_err; }
+
+namespace {
+
+struct DeviceScope {   // make the handle's device current for the call
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceScope(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceScope()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// the handle
+// ---------------------------------------------------------------------------
+
+struct asyncmesh {
+    uint32_t R = 0, S = 0, tau = 0;
+    double p = 0, ema_beta = 0, lr = 0, beta1 = 0, beta2 = 0, eps = 0, wd = 0;
+    uint64_t seed = 0;
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    asyncmesh_alloc_fn alloc = nullptr;
+    asyncmesh_free_fn dealloc = nullptr;
+    void *alloc_ctx = nullptr;
+
+    std::vector<uint64_t> numel, stride;
+    std::vector<uint32_t> delay;
+    std::vector<StageDesc> sd;        // host copy of the stage table
+    std::vector<float *> gstage;      // staging gradients for asyncmesh_step_host
+    std::vector<void *> owned;        // everything obtained from the allocator
+
+    StageDesc *sd_dev = nullptr;
+    unsigned int *cursors = nullptr;  // [n_slots][S]
+    int *status = nullptr;
+    double *scratch = nullptr;        // one double for reductions
+
+    int mode = kSync;
+    uint32_t n_slots = 0;
+    uint32_t total_chunks = 0;
+    int grid = 0;
+    SubsetRule rule{};
+    uint64_t t = 0;
+    uint64_t last_bytes = 0;
+};
+
+static void *dev_alloc(asyncmesh *h, size_t bytes)
+{
+    if (bytes == 0) bytes = 256;
+    void *ptr = nullptr;
+    if (h->alloc) {
+        ptr = h->alloc(h->alloc_ctx, bytes);
+    } else if (cudaMalloc(&ptr, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        ptr = nullptr;
+    }
+    if (ptr) h->owned.push_back(ptr);
+    return ptr;
+}
+
+static void dev_free(asyncmesh *h, void *ptr)
+{
+    if (!ptr) return;
+    for (size_t k = 0; k < h->owned.size(); ++k)
+        if (h->owned[k] == ptr) {
+            h->owned.erase(h->owned.begin() + k);
+            break;
+        }
+    if (h->dealloc) h->dealloc(h->alloc_ctx, ptr);
+    else cudaFree(ptr);
+}
+
+static void release_all(asyncmesh *h)
+{
+    while (!h->owned.empty()) dev_free(h, h->owned.back());
+}
+
+// ---------------------------------------------------------------------------
+// small kernels
+// ---------------------------------------------------------------------------
+
+__global__ void subset_bitmap_kernel(SubsetRule rule, uint32_t stage, uint32_t step, uint64_t N,
+                                     uint8_t *bitmap)
+{
+    const uint64_t nbytes = (N + 7) / 8;
+    for (uint64_t b = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nbytes;
+         b += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t mu = b * 8;
+        uint32_t bits = subset_bits(rule, stage, step, (uint32_t)(mu >> 2));
+        if (mu + 4 < N) bits |= subset_bits(rule, stage, step, (uint32_t)((mu + 4) >> 2)) << 4;
+        const uint64_t left = N - mu;
+        if (left < 8) bits &= (1u << (uint32_t)left) - 1u;
+        bitmap[b] = (uint8_t)bits;
+    }
+}
+
+// dst[mu] = D[mu][i]   (D is coordinate-major)
+__global__ void gather_column_kernel(const float *D, uint32_t R, uint32_t i, uint64_t N, float *dst)
+{
+    for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
+         mu += (uint64_t)gridDim.x * blockDim.x)
+        dst[mu] = D[mu * R + i];
+}
+
+// Replica mean in replica order, one division by (float) R.
+__global__ void mean_rows_kernel(const float *W, uint32_t R, uint64_t stride, uint64_t N, float Rf,
+                                 float *dst)
+{
+    for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
+         mu += (uint64_t)gridDim.x * blockDim.x) {
+        float a = W[mu];
+        for (uint32_t i = 1; i < R; ++i) a = __fadd_rn(a, W[(uint64_t)i * stride + mu]);
+        dst[mu] = __fdiv_rn(a, Rf);
+    }
+}
+
+// sum over coordinates and replicas of (w_i - mean)^2, in double.
+__global__ void consensus_kernel(const float *W, uint32_t R, uint64_t stride, uint64_t N,
+                                 double *out)
+{
+    double acc = 0.0;
+    for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
+         mu += (uint64_t)gridDim.x * blockDim.x) {
+        double mean = 0.0;
+        for (uint32_t i = 0; i < R; ++i) mean += (double)W[(uint64_t)i * stride + mu];
+        mean /= (double)R;
+        for (uint32_t i = 0; i < R; ++i) {
+            const double e = (double)W[(uint64_t)i * stride + mu] - mean;
+            acc += e * e;
+        }
+    }
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+    __shared__ double part[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) part[warp] = acc;
+    __syncthreads();
+    if (warp == 0) {
+        acc = lane < (int)(blockDim.x >> 5) ? part[lane] : 0.0;
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+        if (lane == 0) atomicAdd(out, acc);
+    }
+}
+
+__global__ void philox_debug_kernel(const uint32_t *ctr, const uint32_t *key, uint32_t *out,
+                                    uint64_t n)
+{
+    for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n;
+         k += (uint64_t)gridDim.x * blockDim.x) {
+        const PhiloxOut o = philox4x32_10(ctr[4 * k], ctr[4 * k + 1], ctr[4 * k + 2],
+                                          ctr[4 * k + 3], key[2 * k], key[2 * k + 1]);
+        for (int j = 0; j < 4; ++j) out[4 * k + j] = o.x[j];
+    }
+}
+
+static int grid_for(uint64_t items, int threads)
+{
+    uint64_t blocks = (items + threads - 1) / threads;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148ull * 16) blocks = 148ull * 16;
+    return (int)blocks;
+}
+
+// ---------------------------------------------------------------------------
+// kernel dispatch
+// ---------------------------------------------------------------------------
+
+typedef void (*step_fn)(const StepParams);
+
+template <int R>
+static step_fn pick_mode(int mode)
+{
+    switch (mode) {
+    case kSync: return asyncmesh_step_kernel<R, kSync>;
+    case kCompact: return asyncmesh_step_kernel<R, kCompact>;
+    default: return asyncmesh_step_kernel<R, kDense>;
+    }
+}
+
+static step_fn pick_kernel(uint32_t R, int mode)
+{
+    switch (R) {
+    case 1: return pick_mode<1>(mode);
+    case 2: return pick_mode<2>(mode);
+    case 3: return pick_mode<3>(mode);
+    case 4: return pick_mode<4>(mode);
+    case 5: return pick_mode<5>(mode);
+    case 6: return pick_mode<6>(mode);
+    case 7: return pick_mode<7>(mode);
+    case 8: return pick_mode<8>(mode);
+    case 9: return pick_mode<9>(mode);
+    case 10: return pick_mode<10>(mode);
+    case 11: return pick_mode<11>(mode);
+    case 12: return pick_mode<12>(mode);
+    case 13: return pick_mode<13>(mode);
+    case 14: return pick_mode<14>(mode);
+    case 15: return pick_mode<15>(mode);
+    case 16: return pick_mode<16>(mode);
+    default: return nullptr;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// create / destroy
+// ---------------------------------------------------------------------------
+
+static uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
+
+extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
+{
+    if (out) *out = nullptr;
+    if (!cfg || !out) return fail(ASYNCMESH_ERR_INVALID_ARG, "create: cfg and out must be non-NULL");
+    if (cfg->R < 1 || cfg->R > ASYNCMESH_MAX_REPLICAS)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: R = %u outside 1..%u", cfg->R,
+                    ASYNCMESH_MAX_REPLICAS);
+    if (cfg->S < 1 || cfg->S > ASYNCMESH_MAX_STAGES)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: S = %u outside 1..%u", cfg->S,
+                    ASYNCMESH_MAX_STAGES);
+    if (!cfg->stage_numel) return fail(ASYNCMESH_ERR_INVALID_ARG, "create: stage_numel is NULL");
+    if (!(cfg->p >= 0.0 && cfg->p <= 1.0))
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: p = %g outside [0, 1]", cfg->p);
+    if (cfg->tau > ASYNCMESH_MAX_TAU)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: tau = %u above %u", cfg->tau,
+                    ASYNCMESH_MAX_TAU);
+    if (!(cfg->ema_beta >= 0.0 && cfg->ema_beta <= 1.0))
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: ema_beta = %g outside [0, 1]", cfg->ema_beta);
+    if (!(cfg->lr > 0.0) || !(cfg->eps > 0.0) || !(cfg->weight_decay >= 0.0))
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: need lr > 0, eps > 0, weight_decay >= 0");
+    if (!(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0))
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: betas must lie in [0, 1)");
+    if ((cfg->flags & ~ASYNCMESH_FLAG_SMALL_RING) != 0 || cfg->reserved != 0)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags, or reserved is not 0");
+    if ((cfg->alloc == nullptr) != (cfg->free == nullptr))
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: give both alloc and free, or neither");
+    for (uint32_t s = 0; s < cfg->S; ++s)
+        if (cfg->stage_numel[s] < 1 || cfg->stage_numel[s] > 0xFFFFFFFFull)
+            return fail(ASYNCMESH_ERR_INVALID_ARG, "create: stage_numel[%u] outside 1..2^32-1", s);
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+        cudaGetLastError();
+        return fail(ASYNCMESH_ERR_CUDA, "create: no CUDA device is usable (there is no CPU path)");
+    }
+    if (cfg->device < 0 || cfg->device >= ndev)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: device %d outside 0..%d", cfg->device, ndev - 1);
+
+    DeviceScope scope(cfg->device);
+    if (!scope.ok) return fail(ASYNCMESH_ERR_CUDA, "create: cudaSetDevice(%d) failed", cfg->device);
+
+    asyncmesh *h = new (std::nothrow) asyncmesh();
+    if (!h) return fail(ASYNCMESH_ERR_OOM, "create: host allocation failed");
+    h->R = cfg->R; h->S = cfg->S; h->tau = cfg->tau;
+    h->p = cfg->p; h->ema_beta = cfg->ema_beta; h->lr = cfg->lr;
+    h->beta1 = cfg->beta1; h->beta2 = cfg->beta2; h->eps = cfg->eps; h->wd = cfg->weight_decay;
+    h->seed = cfg->seed; h->device = cfg->device; h->stream = (cudaStream_t)cfg->stream;
+    h->alloc = cfg->alloc; h->dealloc = cfg->free; h->alloc_ctx = cfg->alloc_ctx;
+
+    const uint32_t R = h->R, S = h->S;
+    h->numel.assign(cfg->stage_numel, cfg->stage_numel + S);
+    h->stride.resize(S);
+    h->delay.resize(S);
+    h->sd.assign(S, StageDesc{});
+    h->gstage.assign(S, nullptr);
+
+    // subset rule: floor(p * 2^32) in double
+    const double tf = std::floor(cfg->p * 4294967296.0);
+    h->rule.key0 = (uint32_t)h->seed;
+    h->rule.key1 = (uint32_t)(h->seed >> 32);
+    if (tf >= 4294967296.0) { h->rule.mode = 1; h->rule.thresh = 0xFFFFFFFFu; }
+    else if (tf <= 0.0) { h->rule.mode = 2; h->rule.thresh = 0; }
+    else { h->rule.mode = 0; h->rule.thresh = (uint32_t)tf; }
+
+    // ring layout: compact unless it would not be smaller than dense
+    std::vector<uint64_t> cap(S);
+    long double compact_total = 0, dense_total = 0;
+    uint64_t chunks = 0;
+    for (uint32_t s = 0; s < S; ++s) {
+        const uint64_t N = h->numel[s];
+        h->stride[s] = round_up(N, 32);
+        h->delay[s] = cfg->lookahead_delay ? cfg->lookahead_delay[s] : (S - 1 - s);
+        const double mean = cfg->p * (double)N;
+        const double sd = std::sqrt(mean * (1.0 - cfg->p));
+        double c = std::ceil(mean + 8.0 * sd) + 64.0;   // 8 sigma: never reached in practice
+        if (c > (double)N) c = (double)N;
+        cap[s] = (uint64_t)c;
+        if ((cfg->flags & ASYNCMESH_FLAG_SMALL_RING) && h->tau > 0) cap[s] = cap[s] / 8 + 1;
+        compact_total += (long double)(h->tau + 1) * cap[s];
+        dense_total += (long double)h->tau * h->stride[s];
+        h->sd[s].n_chunks = (uint32_t)((N + kWarpChunk - 1) / kWarpChunk);
+        h->sd[s].chunk_begin = (uint32_t)chunks;
+        chunks += h->sd[s].n_chunks;
+    }
+    if (chunks > 0xFFFFFFF0ull) {
+        delete h;
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: too many coordinates in total");
+    }
+    h->total_chunks = (uint32_t)chunks;
+    if (h->tau == 0) { h->mode = kSync; h->n_slots = 0; }
+    else if (dense_total <= compact_total && !(cfg->flags & ASYNCMESH_FLAG_SMALL_RING)) {
+        h->mode = kDense; h->n_slots = h->tau;
+    }
+    else { h->mode = kCompact; h->n_slots = h->tau + 1; }
+
+    auto bail = [&](int code, const char *what) {
+        release_all(h);
+        delete h;
+        return fail(code, "create: %s", what);
+    };
+
+    // allocations (all zeroed on the stream)
+    auto zalloc = [&](size_t bytes) -> void * {
+        void *ptr = dev_alloc(h, bytes);
+        if (ptr && cudaMemsetAsync(ptr, 0, bytes ? bytes : 256, h->stream) != cudaSuccess) return nullptr;
+        return ptr;
+    };
+    for (uint32_t s = 0; s < S; ++s) {
+        StageDesc &d = h->sd[s];
+        const size_t row_bytes = (size_t)R * h->stride[s] * sizeof(float);
+        d.N = h->numel[s];
+        d.stride = h->stride[s];
+        d.stage_id = s;
+        d.delta = (float)h->delay[s];
+        d.has_look = h->delay[s] != 0 ? 1u : 0u;
+        d.cap = (uint32_t)cap[s];
+        d.W = (float *)zalloc(row_bytes);
+        d.M = (float *)zalloc(row_bytes);
+        d.V = (float *)zalloc(row_bytes);
+        d.D = (float *)zalloc(row_bytes);
+        if (!d.W || !d.M || !d.V || !d.D) return bail(ASYNCMESH_ERR_OOM, "out of device memory (state)");
+        d.LOOK = d.W;
+        if (d.has_look) {
+            d.LOOK = (float *)zalloc(row_bytes);
+            if (!d.LOOK) return bail(ASYNCMESH_ERR_OOM, "out of device memory (look-ahead)");
+        }
+        if (h->mode == kCompact) {
+            d.slot_floats = round_up(cap[s] * R, 64);
+            d.chunk_base = (uint32_t *)zalloc((size_t)h->n_slots * d.n_chunks * sizeof(uint32_t));
+            if (!d.chunk_base) return bail(ASYNCMESH_ERR_OOM, "out of device memory (ring index)");
+        } else if (h->mode == kDense) {
+            d.slot_floats = h->stride[s] * R;
+        }
+        if (h->mode != kSync) {
+            d.ring = (float *)zalloc((size_t)h->n_slots * d.slot_floats * sizeof(float));
+            if (!d.ring) return bail(ASYNCMESH_ERR_OOM, "out of device memory (snapshot ring)");
+        }
+    }
+    h->sd_dev = (StageDesc *)zalloc(S * sizeof(StageDesc));
+    h->cursors = (unsigned int *)zalloc((size_t)(h->n_slots + 1) * S * sizeof(unsigned int));
+    h->status = (int *)zalloc(256);
+    h->scratch = (double *)zalloc(256);
+    if (!h->sd_dev || !h->cursors || !h->status || !h->scratch)
+        return bail(ASYNCMESH_ERR_OOM, "out of device memory (tables)");
+    if (cudaMemcpyAsync(h->sd_dev, h->sd.data(), S * sizeof(StageDesc), cudaMemcpyHostToDevice,
+                        h->stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->stream) != cudaSuccess) {
+        const char *msg = cudaGetErrorString(cudaGetLastError());
+        release_all(h);
+        delete h;
+        return fail(ASYNCMESH_ERR_CUDA, "create: uploading the stage table failed: %s", msg);
+    }
+
+    // persistent grid: every SM filled to the kernel's occupancy
+    step_fn fn = pick_kernel(R, h->mode);
+    int sms = 0, per_sm = 0;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kBlockThreads, 0) != cudaSuccess ||
+        per_sm < 1 || sms < 1) {
+        const char *msg = cudaGetErrorString(cudaGetLastError());
+        release_all(h);
+        delete h;
+        return fail(ASYNCMESH_ERR_CUDA, "create: the step kernel cannot run on this device: %s", msg);
+    }
+    uint64_t blocks = (uint64_t)sms * per_sm;
+    const uint64_t need = ((uint64_t)h->total_chunks + kBlockThreads / 32 - 1) / (kBlockThreads / 32);
+    if (blocks > need) blocks = need;
+    h->grid = (int)blocks;
+
+    *out = h;
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_destroy(asyncmesh *h)
+{
+    if (!h) return ASYNCMESH_OK;
+    DeviceScope scope(h->device);
+    cudaStreamSynchronize(h->stream);
+    release_all(h);
+    delete h;
+    return ASYNCMESH_OK;
+}
+
+// ---------------------------------------------------------------------------
+// parameters in
+// ---------------------------------------------------------------------------
+
+extern "C" int asyncmesh_init_params(asyncmesh *h, uint32_t stage, int32_t replica,
+                                     const float *src, uint64_t n, int src_on_device)
+{
+    if (!h || !src) return fail(ASYNCMESH_ERR_INVALID_ARG, "init_params: NULL argument");
+    if (stage >= h->S) return fail(ASYNCMESH_ERR_INVALID_ARG, "init_params: stage %u >= S", stage);
+    if (replica < -1 || replica >= (int32_t)h->R)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "init_params: replica %d outside -1..R-1", replica);
+    if (n != h->numel[stage])
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "init_params: n = %llu, stage holds %llu",
+                    (unsigned long long)n, (unsigned long long)h->numel[stage]);
+    if (h->t != 0) return fail(ASYNCMESH_ERR_BAD_STATE, "init_params: steps were already taken");
+    DeviceScope scope(h->device);
+    const StageDesc &d = h->sd[stage];
+    const cudaMemcpyKind kind = src_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    for (uint32_t i = 0; i < h->R; ++i) {
+        if (replica >= 0 && (uint32_t)replica != i) continue;
+        CU_TRY(cudaMemcpyAsync(d.W + (uint64_t)i * d.stride, src, n * sizeof(float), kind, h->stream));
+        if (d.has_look)
+            CU_TRY(cudaMemcpyAsync(d.LOOK + (uint64_t)i * d.stride, src, n * sizeof(float), kind,
+                                   h->stream));
+    }
+    if (!src_on_device) CU_TRY(cudaStreamSynchronize(h->stream));
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_row_stride(const asyncmesh *h, uint32_t stage, uint64_t *stride)
+{
+    if (!h || !stride || stage >= h->S)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "row_stride: bad handle, stage or output");
+    *stride = h->stride[stage];
+    return ASYNCMESH_OK;
+}
+
+// ---------------------------------------------------------------------------
+// the step
+// ---------------------------------------------------------------------------
+
+static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_t, double lr_t)
+{
+    if (ema_beta_t > 1.0) return fail(ASYNCMESH_ERR_INVALID_ARG, "step: ema_beta_t = %g above 1", ema_beta_t);
+    StepParams P;
+    std::memset(&P, 0, sizeof(P));
+    for (uint32_t s = 0; s < h->S; ++s) {
+        if (!grads[s]) return fail(ASYNCMESH_ERR_INVALID_ARG, "step: grads[%u] is NULL", s);
+        if (((uintptr_t)grads[s] & 15u) != 0)
+            return fail(ASYNCMESH_ERR_INVALID_ARG, "step: grads[%u] is not 16-byte aligned", s);
+        P.G[s] = grads[s];
+    }
+    const uint64_t t = h->t + 1;
+    const double lam = ema_beta_t >= 0.0 ? ema_beta_t : h->ema_beta;
+    const double lr = lr_t >= 0.0 ? lr_t : h->lr;
+
+    P.stages = h->sd_dev;
+    P.cursors = h->cursors;
+    P.status = h->status;
+    P.S = h->S;
+    P.total_chunks = h->total_chunks;
+    P.step = (uint32_t)t;
+    P.cons_step = (uint32_t)(t - h->tau);
+    P.consume = (h->mode != kSync && t > h->tau) ? 1u : 0u;
+    if (h->mode == kCompact) {
+        P.prod_slot = (uint32_t)(t % (h->tau + 1));
+        P.cons_slot = (uint32_t)((t - h->tau) % (h->tau + 1));   // unused while t <= tau
+    } else if (h->mode == kDense) {
+        P.prod_slot = P.cons_slot = (uint32_t)(t % h->tau);
+    }
+    P.rule = h->rule;
+    // per-step scalars: double arithmetic, one rounding to fp32 each
+    P.b1 = (float)h->beta1;
+    P.b2 = (float)h->beta2;
+    P.omb1 = (float)(1.0 - h->beta1);
+    P.omb2 = (float)(1.0 - h->beta2);
+    P.ib1 = (float)(1.0 / (1.0 - std::pow(h->beta1, (double)t)));
+    P.ib2 = (float)(1.0 / (1.0 - std::pow(h->beta2, (double)t)));
+    P.eps = (float)h->eps;
+    P.lr = (float)lr;
+    P.lrwd = (float)(lr * h->wd);
+    P.lam = (float)lam;
+    P.oml = (float)(1.0 - lam);
+    P.Rf = (float)h->R;
+
+    if (h->mode == kCompact)   // the producing slot's cursors start this step at zero
+        CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
+                               h->S * sizeof(unsigned int), h->stream));
+
+    step_fn fn = pick_kernel(h->R, h->mode);
+    fn<<<h->grid, kBlockThreads, 0, h->stream>>>(P);
+    CU_TRY(cudaGetLastError());
+    h->t = t;
+
+    // roofline numerator (see the header): bytes this step could not avoid
+    double bytes = 0.0;
+    for (uint32_t s = 0; s < h->S; ++s) {
+        double per = 28.0 + (h->delay[s] ? 4.0 : 0.0);
+        if (h->mode != kSync) per += 4.0 * h->p + (P.consume ? 12.0 * h->p : 0.0);
+        bytes += per * (double)h->R * (double)h->numel[s];
+    }
+    h->last_bytes = (uint64_t)bytes;
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_step_ex(asyncmesh *h, const float *const *grads, double ema_beta_t,
+                                 double lr_t)
+{
+    if (!h || !grads) return fail(ASYNCMESH_ERR_INVALID_ARG, "step: NULL argument");
+    DeviceScope scope(h->device);
+    return launch_step(h, grads, ema_beta_t, lr_t);
+}
+
+extern "C" int asyncmesh_step(asyncmesh *h, const float *const *grads)
+{
+    return asyncmesh_step_ex(h, grads, -1.0, -1.0);
+}
+
+extern "C" int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host)
+{
+    if (!h || !grads_host) return fail(ASYNCMESH_ERR_INVALID_ARG, "step_host: NULL argument");
+    DeviceScope scope(h->device);
+    for (uint32_t s = 0; s < h->S; ++s) {
+        if (!grads_host[s]) return fail(ASYNCMESH_ERR_INVALID_ARG, "step_host: grads_host[%u] is NULL", s);
+        if (!h->gstage[s]) {
+            const size_t bytes = (size_t)h->R * h->stride[s] * sizeof(float);
+            h->gstage[s] = (float *)dev_alloc(h, bytes);
+            if (!h->gstage[s]) return fail(ASYNCMESH_ERR_OOM, "step_host: out of device memory (staging)");
+            CU_TRY(cudaMemsetAsync(h->gstage[s], 0, bytes, h->stream));
+        }
+        const size_t n = h->numel[s] * sizeof(float);
+        CU_TRY(cudaMemcpy2DAsync(h->gstage[s], h->stride[s] * sizeof(float), grads_host[s], n, n,
+                                 h->R, cudaMemcpyHostToDevice, h->stream));
+    }
+    return launch_step(h, h->gstage.data(), -1.0, -1.0);
+}
+
+// ---------------------------------------------------------------------------
+// results out
+// ---------------------------------------------------------------------------
+
+static int check_status(asyncmesh *h, const char *who)
+{
+    int st = 0;
+    CU_TRY(cudaMemcpyAsync(&st, h->status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+    CU_TRY(cudaStreamSynchronize(h->stream));
+    if (st == kStatusRingOverflow)
+        return fail(ASYNCMESH_ERR_DEVICE_STATUS,
+                    "%s: a snapshot ring slot overflowed its capacity; results are invalid", who);
+    if (st != 0) return fail(ASYNCMESH_ERR_DEVICE_STATUS, "%s: device status %d", who, st);
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_status(asyncmesh *h)
+{
+    if (!h) return fail(ASYNCMESH_ERR_INVALID_ARG, "status: NULL handle");
+    DeviceScope scope(h->device);
+    return check_status(h, "status");
+}
+
+extern "C" int asyncmesh_lookahead_weights(asyncmesh *h, uint32_t stage, uint32_t delay,
+                                           const float **out_device, uint64_t *row_stride)
+{
+    if (!h || !out_device || !row_stride || stage >= h->S)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "lookahead_weights: bad handle, stage or output");
+    const StageDesc &d = h->sd[stage];
+    if (delay == 0) *out_device = d.W;
+    else if (delay == h->delay[stage]) *out_device = d.LOOK;
+    else
+        return fail(ASYNCMESH_ERR_UNSUPPORTED,
+                    "lookahead_weights: stage %u was configured with delay %u, not %u", stage,
+                    h->delay[stage], delay);
+    *row_stride = d.stride;
+    return ASYNCMESH_OK;
+}
+
+// Copy N floats produced on the device (by `produce`, into a device buffer) to dst.
+template <typename Produce>
+static int deliver(asyncmesh *h, float *dst, uint64_t n, int dst_on_device, Produce produce)
+{
+    float *tmp = dst;
+    if (!dst_on_device) {
+        tmp = (float *)dev_alloc(h, n * sizeof(float));
+        if (!tmp) return fail(ASYNCMESH_ERR_OOM, "read: out of device memory (temporary)");
+    }
+    produce(tmp);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && !dst_on_device)
+        e = cudaMemcpyAsync(dst, tmp, n * sizeof(float), cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (!dst_on_device) dev_free(h, tmp);
+    if (e != cudaSuccess) return fail(ASYNCMESH_ERR_CUDA, "read: %s", cudaGetErrorString(e));
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_read_state(asyncmesh *h, uint32_t stage, int which, int32_t replica,
+                                    float *dst, uint64_t n, int dst_on_device)
+{
+    if (!h || !dst) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: NULL argument");
+    if (stage >= h->S) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: stage %u >= S", stage);
+    if (replica < 0 || replica >= (int32_t)h->R)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: replica %d outside 0..R-1", replica);
+    if (n != h->numel[stage])
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: n = %llu, stage holds %llu",
+                    (unsigned long long)n, (unsigned long long)h->numel[stage]);
+    DeviceScope scope(h->device);
+    int rc = check_status(h, "read_state");
+    if (rc != ASYNCMESH_OK) return rc;
+    const StageDesc &d = h->sd[stage];
+    const float *row = nullptr;
+    switch (which) {
+    case ASYNCMESH_STATE_W: row = d.W; break;
+    case ASYNCMESH_STATE_M: row = d.M; break;
+    case ASYNCMESH_STATE_V: row = d.V; break;
+    case ASYNCMESH_STATE_LOOK: row = d.LOOK; break;
+    case ASYNCMESH_STATE_D: break;
+    default: return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: unknown selector %d", which);
+    }
+    if (row) {
+        CU_TRY(cudaMemcpyAsync(dst, row + (uint64_t)replica * d.stride, n * sizeof(float),
+                               dst_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost,
+                               h->stream));
+        CU_TRY(cudaStreamSynchronize(h->stream));
+        return ASYNCMESH_OK;
+    }
+    return deliver(h, dst, n, dst_on_device, [&](float *out) {
+        gather_column_kernel<<<grid_for(n, 256), 256, 0, h->stream>>>(d.D, h->R, (uint32_t)replica, n, out);
+    });
+}
+
+extern "C" int asyncmesh_read_params(asyncmesh *h, uint32_t stage, int32_t replica, float *dst,
+                                     uint64_t n, int dst_on_device)
+{
+    if (!h || !dst) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_params: NULL argument");
+    if (replica >= 0) return asyncmesh_read_state(h, stage, ASYNCMESH_STATE_W, replica, dst, n, dst_on_device);
+    if (replica != -1) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_params: replica %d outside -1..R-1", replica);
+    if (stage >= h->S) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_params: stage %u >= S", stage);
+    if (n != h->numel[stage])
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "read_params: n = %llu, stage holds %llu",
+                    (unsigned long long)n, (unsigned long long)h->numel[stage]);
+    DeviceScope scope(h->device);
+    int rc = check_status(h, "read_params");
+    if (rc != ASYNCMESH_OK) return rc;
+    const StageDesc &d = h->sd[stage];
+    return deliver(h, dst, n, dst_on_device, [&](float *out) {
+        mean_rows_kernel<<<grid_for(n, 256), 256, 0, h->stream>>>(d.W, h->R, d.stride, n, (float)h->R, out);
+    });
+}
+
+extern "C" int asyncmesh_subset_mask(asyncmesh *h, uint32_t stage, uint64_t step,
+                                     uint8_t *bitmap_host)
+{
+    if (!h || !bitmap_host || stage >= h->S)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "subset_mask: bad handle, stage or output");
+    DeviceScope scope(h->device);
+    const uint64_t N = h->numel[stage], nbytes = (N + 7) / 8;
+    uint8_t *tmp = (uint8_t *)dev_alloc(h, nbytes);
+    if (!tmp) return fail(ASYNCMESH_ERR_OOM, "subset_mask: out of device memory (temporary)");
+    subset_bitmap_kernel<<<grid_for(nbytes, 256), 256, 0, h->stream>>>(h->rule, stage, (uint32_t)step, N, tmp);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemcpyAsync(bitmap_host, tmp, nbytes, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    dev_free(h, tmp);
+    if (e != cudaSuccess) return fail(ASYNCMESH_ERR_CUDA, "subset_mask: %s", cudaGetErrorString(e));
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *out_host)
+{
+    if (!h || !out_host || stage >= h->S)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "consensus_error: bad handle, stage or output");
+    DeviceScope scope(h->device);
+    const StageDesc &d = h->sd[stage];
+    CU_TRY(cudaMemsetAsync(h->scratch, 0, sizeof(double), h->stream));
+    consensus_kernel<<<grid_for(d.N, 256), 256, 0, h->stream>>>(d.W, h->R, d.stride, d.N, h->scratch);
+    CU_TRY(cudaGetLastError());
+    CU_TRY(cudaMemcpyAsync(out_host, h->scratch, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+    CU_TRY(cudaStreamSynchronize(h->stream));
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_step_count(const asyncmesh *h, uint64_t *t)
+{
+    if (!h || !t) return fail(ASYNCMESH_ERR_INVALID_ARG, "step_count: NULL argument");
+    *t = h->t;
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_min_bytes_last_step(const asyncmesh *h, uint64_t *bytes)
+{
+    if (!h || !bytes) return fail(ASYNCMESH_ERR_INVALID_ARG, "min_bytes_last_step: NULL argument");
+    *bytes = h->last_bytes;
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_debug_philox(int device, const uint32_t *ctr_host, const uint32_t *key_host,
+                                      uint32_t *out_host, uint64_t n)
+{
+    if (!ctr_host || !key_host || !out_host) return fail(ASYNCMESH_ERR_INVALID_ARG, "debug_philox: NULL argument");
+    if (n == 0) return ASYNCMESH_OK;
+    DeviceScope scope(device);
+    if (!scope.ok) return fail(ASYNCMESH_ERR_CUDA, "debug_philox: cudaSetDevice(%d) failed", device);
+    uint32_t *c = nullptr, *k = nullptr, *o = nullptr;
+    cudaError_t e = cudaMalloc(&c, n * 16);
+    if (e == cudaSuccess) e = cudaMalloc(&k, n * 8);
+    if (e == cudaSuccess) e = cudaMalloc(&o, n * 16);
+    if (e == cudaSuccess) e = cudaMemcpy(c, ctr_host, n * 16, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(k, key_host, n * 8, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+        philox_debug_kernel<<<grid_for(n, 256), 256>>>(c, k, o, n);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(out_host, o, n * 16, cudaMemcpyDeviceToHost);
+    cudaFree(c); cudaFree(k); cudaFree(o);
+    if (e != cudaSuccess) return fail(ASYNCMESH_ERR_CUDA, "debug_philox: %s", cudaGetErrorString(e));
+    return ASYNCMESH_OK;
+}

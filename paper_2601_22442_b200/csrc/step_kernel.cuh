@@ -1,0 +1,367 @@
+// The fused AsyncMesh step for sm_100a: one launch advances every stage of the
+// mesh by one step.  HBM-bound streaming kernel: per replica-coordinate it reads
+// w, g, m, v once (128-bit loads) and writes w, m, v (and the look-ahead) once;
+// the sparse parts (snapshot ring, EMA state d) are touched only at selected
+// coordinates.  No tensor cores: there is no contraction on this path.
+//
+// Work decomposition.  A stage's coordinates are cut into warp chunks of 1024
+// (8 sub-iterations x 32 lanes x 4 coordinates).  A warp owns a chunk, so a
+// lane sees, per sub-iteration, one float4 of every array row of every replica.
+// All chunks of all stages form one list that the grid's warps walk with a
+// grid-sized stride, so neighbouring warps stream neighbouring 4 KB pieces.
+//
+// Snapshot ring (Section 3.1: the average of step t is consumed at t + tau; the
+// paper's own experiments buffer it).  A slot holds, for one step u, the local
+// iterates w^_i^u of the coordinates in S^u, coordinate-major: R floats per
+// selected coordinate.  Two layouts:
+//   compact  slot = [cap][R]; a warp reserves room for its chunk's selected
+//            coordinates with one atomicAdd on the slot's cursor and records the
+//            base in chunk_base[slot][chunk]; tau steps later the consumer finds
+//            the data through that table and recomputes membership and rank
+//            from Philox, so no index list is stored.  tau + 1 slots.
+//   dense    slot = [row_stride][R], coordinate mu at position mu; used when the
+//            subset is so large that compaction saves nothing.  tau slots; the
+//            consumer and producer of a step share a slot and a thread reads a
+//            position before it overwrites it.
+// With tau = 0 (synchronous sparse averaging, Eq. "sparta") there is no ring:
+// the average is formed from the registers of the lane that owns the coordinate.
+//
+// Arithmetic is written with the round-to-nearest intrinsics, one IEEE
+// operation per paper operation, so that no contraction into FMA can change a
+// result; the same operation order is what the CPU check uses.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "philox.cuh"
+
+namespace amk {
+
+constexpr int kWarpChunk = 1024;   // coordinates a warp owns at a time
+constexpr int kSubIters = 8;       // 8 x (32 lanes x 4 coordinates)
+constexpr int kBlockThreads = 256;
+constexpr uint32_t kInvalidBase = 0xFFFFFFFFu;
+constexpr unsigned kFullMask = 0xFFFFFFFFu;
+constexpr int kMaxStages = 64;
+
+enum RingMode : int { kSync = 0, kCompact = 1, kDense = 2 };
+
+constexpr int kStatusRingOverflow = 1;
+
+struct StageDesc {
+    float *W, *M, *V;       // [R][stride]
+    float *D;               // [stride][R]
+    float *LOOK;            // [R][stride]; == W when delta == 0
+    float *ring;            // [n_slots][slot_floats]
+    uint32_t *chunk_base;   // [n_slots][n_chunks]           (compact only)
+    uint64_t N, stride, slot_floats;
+    uint32_t n_chunks;      // ceil(N / 1024)
+    uint32_t chunk_begin;   // first chunk of this stage in the global list
+    uint32_t cap;           // selected coordinates a compact slot can hold
+    uint32_t stage_id;
+    float delta;            // look-ahead delay as a float
+    uint32_t has_look;      // LOOK is a buffer of its own
+};
+
+struct StepParams {
+    const StageDesc *stages;     // device [S]
+    unsigned int *cursors;       // device [n_slots][S]            (compact only)
+    int *status;                 // device status word
+    const float *G[kMaxStages];  // gradients, [R][stride] each
+    uint32_t S, total_chunks;
+    uint32_t step, cons_step;    // t and t - tau
+    uint32_t consume;            // t > tau
+    uint32_t prod_slot, cons_slot;
+    SubsetRule rule;
+    float b1, b2, omb1, omb2, ib1, ib2, eps, lr, lrwd, lam, oml, Rf;
+};
+
+__device__ __forceinline__ float4 ld_stream(const float *p)
+{
+    return __ldcs(reinterpret_cast<const float4 *>(p));
+}
+__device__ __forceinline__ void st_stream(float *p, const float (&x)[4])
+{
+    __stcs(reinterpret_cast<float4 *>(p), make_float4(x[0], x[1], x[2], x[3]));
+}
+
+// AdamW with decoupled weight decay and bias correction, one rounding per
+// written operation (first line of Eq. "sparta": the local optimizer step).
+__device__ __forceinline__ void adamw(const StepParams &P, float w, float g, float &m,
+                                      float &v, float &what)
+{
+    m = __fadd_rn(__fmul_rn(P.b1, m), __fmul_rn(P.omb1, g));
+    v = __fadd_rn(__fmul_rn(P.b2, v), __fmul_rn(P.omb2, __fmul_rn(g, g)));
+    const float mh = __fmul_rn(m, P.ib1);
+    const float vh = __fmul_rn(v, P.ib2);
+    const float den = __fadd_rn(__fsqrt_rn(vh), P.eps);
+    const float u = __fdiv_rn(mh, den);
+    const float decayed = __fsub_rn(w, __fmul_rn(P.lrwd, w));
+    what = __fsub_rn(decayed, __fmul_rn(P.lr, u));
+}
+
+template <int R>
+__device__ __forceinline__ void load_replicas(const float *p, float (&x)[R])
+{
+    if constexpr (R % 4 == 0) {
+#pragma unroll
+        for (int q = 0; q < R / 4; ++q) {
+            const float4 t = *reinterpret_cast<const float4 *>(p + 4 * q);
+            x[4 * q] = t.x; x[4 * q + 1] = t.y; x[4 * q + 2] = t.z; x[4 * q + 3] = t.w;
+        }
+    } else if constexpr (R % 2 == 0) {
+#pragma unroll
+        for (int q = 0; q < R / 2; ++q) {
+            const float2 t = *reinterpret_cast<const float2 *>(p + 2 * q);
+            x[2 * q] = t.x; x[2 * q + 1] = t.y;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < R; ++i) x[i] = p[i];
+    }
+}
+
+__device__ __forceinline__ uint32_t warp_exclusive_sum(uint32_t x, int lane, uint32_t &total)
+{
+    uint32_t incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t n = __shfl_up_sync(kFullMask, incl, d);
+        if (lane >= d) incl += n;
+    }
+    total = __shfl_sync(kFullMask, incl, 31);
+    return incl - x;
+}
+
+template <int R, int MODE>
+__device__ __forceinline__ void process_chunk(const StepParams &P, const StageDesc &st,
+                                              const float *__restrict__ G, uint32_t s,
+                                              uint32_t chunk, int lane)
+{
+    constexpr int RG = (R % 2 == 0) ? 2 : 1;   // replicas loaded together
+    const uint64_t N = st.N, stride = st.stride;
+    const uint64_t c0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
+    const bool consume = (MODE != kSync) && (P.consume != 0u);
+
+    // ---- membership of this lane's 32 coordinates in S^t and S^{t-tau} --------
+    uint32_t pmask = 0, cmask = 0;   // bit 4k+j: coordinate c0 + 128k + j
+#pragma unroll 2
+    for (int k = 0; k < kSubIters; ++k) {
+        const uint64_t mu = c0 + (uint64_t)k * 128;
+        if (mu < N) {
+            const uint64_t left = N - mu;
+            const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
+            const uint32_t quad = (uint32_t)(mu >> 2);
+            pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * k);
+            if (consume)
+                cmask |= (subset_bits(P.rule, st.stage_id, P.cons_step, quad) & valid) << (4 * k);
+        }
+    }
+
+    // ---- where this chunk's selected coordinates live in the ring slots --------
+    uint32_t pbase = 0, pexcl = 0, cbase = 0, cexcl = 0;
+    if constexpr (MODE == kCompact) {
+        uint32_t total;
+        pexcl = warp_exclusive_sum(__popc(pmask), lane, total);
+        if (lane == 0) {
+            uint32_t b = 0;
+            if (total) {
+                b = atomicAdd(&P.cursors[P.prod_slot * P.S + s], total);
+                if (b > st.cap || total > st.cap - b) {   // slot full: drop loudly
+                    b = kInvalidBase;
+                    atomicExch(P.status, kStatusRingOverflow);
+                }
+            }
+            st.chunk_base[(uint64_t)P.prod_slot * st.n_chunks + chunk] = b;
+            pbase = b;
+        }
+        pbase = __shfl_sync(kFullMask, pbase, 0);
+        if (pbase == kInvalidBase) pmask = 0;
+        if (consume) {
+            cbase = st.chunk_base[(uint64_t)P.cons_slot * st.n_chunks + chunk];
+            if (cbase == kInvalidBase) cmask = 0;
+            uint32_t ctotal;
+            cexcl = warp_exclusive_sum(__popc(cmask), lane, ctotal);
+        }
+    }
+    const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
+    float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
+    const float delta = st.delta;
+    const bool has_look = st.has_look != 0u;
+
+#pragma unroll 1
+    for (int k = 0; k < kSubIters; ++k) {
+        const uint64_t mu = c0 + (uint64_t)k * 128;
+        if (mu >= N) break;   // no warp-wide operation below this point
+        const uint32_t pm = (pmask >> (4 * k)) & 0xFu;
+        const uint32_t cm = (cmask >> (4 * k)) & 0xFu;
+
+        // ---- stale average wbar^{t-tau} of the coordinates being consumed -----
+        float abar[4] = {0.f, 0.f, 0.f, 0.f};
+        uint64_t ce[4] = {0, 0, 0, 0}, pe[4] = {0, 0, 0, 0};   // ring offsets (floats)
+        if constexpr (MODE != kSync) {
+            if (cm) {
+                const uint32_t below = __popc(cmask & ((1u << (4 * k)) - 1u));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if ((cm >> j) & 1u) {
+                        const uint64_t idx = (MODE == kDense)
+                            ? (mu + j)
+                            : (uint64_t)(cbase + cexcl + below + __popc(cm & ((1u << j) - 1u)));
+                        ce[j] = idx * R;
+                        float old[R];
+                        load_replicas<R>(ring_cons + ce[j], old);
+                        float a = old[0];
+#pragma unroll
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, old[i]);
+                        abar[j] = __fdiv_rn(a, P.Rf);
+                    }
+                }
+            }
+            if (pm) {
+                const uint32_t below = __popc(pmask & ((1u << (4 * k)) - 1u));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if ((pm >> j) & 1u) {
+                        const uint64_t idx = (MODE == kDense)
+                            ? (mu + j)
+                            : (uint64_t)(pbase + pexcl + below + __popc(pm & ((1u << j) - 1u)));
+                        pe[j] = idx * R;
+                    }
+                }
+            }
+        }
+
+        float wold_keep[MODE == kSync ? R : 1][4];
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+
+#pragma unroll
+        for (int i0 = 0; i0 < R; i0 += RG) {
+            // -- load phase: everything this group needs, issued back to back --
+            float4 w4[RG], g4[RG], m4[RG], v4[RG];
+            float old[RG][4], dd[RG][4];
+#pragma unroll
+            for (int ii = 0; ii < RG; ++ii) {
+                const uint64_t off = (uint64_t)(i0 + ii) * stride + mu;
+                w4[ii] = ld_stream(st.W + off);
+                g4[ii] = ld_stream(G + off);
+                m4[ii] = ld_stream(st.M + off);
+                v4[ii] = ld_stream(st.V + off);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    old[ii][j] = 0.f;
+                    dd[ii][j] = 0.f;
+                    if constexpr (MODE != kSync) {
+                        if ((cm >> j) & 1u) {
+                            old[ii][j] = ring_cons[ce[j] + (i0 + ii)];
+                            dd[ii][j] = st.D[(mu + j) * R + (i0 + ii)];
+                        }
+                    }
+                }
+            }
+            // -- compute and write back, one replica at a time --
+#pragma unroll
+            for (int ii = 0; ii < RG; ++ii) {
+                const int i = i0 + ii;
+                const uint64_t off = (uint64_t)i * stride + mu;
+                const float w[4] = {w4[ii].x, w4[ii].y, w4[ii].z, w4[ii].w};
+                const float g[4] = {g4[ii].x, g4[ii].y, g4[ii].z, g4[ii].w};
+                float m[4] = {m4[ii].x, m4[ii].y, m4[ii].z, m4[ii].w};
+                float v[4] = {v4[ii].x, v4[ii].y, v4[ii].z, v4[ii].w};
+                float wh[4], wn[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    adamw(P, w[c], g[c], m[c], v[c], wh[c]);
+                    wn[c] = wh[c];
+                }
+                st_stream(st.M + off, m);
+                st_stream(st.V + off, v);
+
+                if constexpr (MODE != kSync) {
+                    // Eq. "ema" + corrected averaging on S^{t-tau}
+                    if (cm) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if ((cm >> j) & 1u) {
+                                const float diff = __fsub_rn(wh[j], old[ii][j]);
+                                const float dn = __fadd_rn(__fmul_rn(P.oml, dd[ii][j]),
+                                                           __fmul_rn(P.lam, diff));
+                                st.D[(mu + j) * R + i] = dn;
+                                wn[j] = __fadd_rn(abar[j], dn);
+                            }
+                        }
+                    }
+                    // snapshot of the local iterate on S^t
+                    if (pm) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if ((pm >> j) & 1u) ring_prod[pe[j] + i] = wh[j];
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        acc[c] = (i == 0) ? wh[c] : __fadd_rn(acc[c], wh[c]);
+                        wold_keep[i][c] = w[c];
+                    }
+                }
+
+                st_stream(st.W + off, wn);
+                if (has_look) {   // Section 2.2: extrapolate the last update direction
+                    float lk[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        lk[c] = __fadd_rn(wn[c], __fmul_rn(delta, __fsub_rn(wn[c], w[c])));
+                    st_stream(st.LOOK + off, lk);
+                }
+            }
+        }
+
+        if constexpr (MODE == kSync) {
+            // Eq. "sparta": coordinates of S^t take the replica mean.  The EMA
+            // state stays exactly zero when tau = 0 (its sample is w^ - w^ = 0),
+            // so the corrected value is mean + 0.
+            if (pm) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if ((pm >> j) & 1u) {
+                        const float wnew = __fadd_rn(__fdiv_rn(acc[j], P.Rf), 0.0f);
+#pragma unroll
+                        for (int i = 0; i < R; ++i) {
+                            const uint64_t o1 = (uint64_t)i * stride + mu + j;
+                            st.W[o1] = wnew;
+                            if (has_look)
+                                st.LOOK[o1] = __fadd_rn(
+                                    wnew, __fmul_rn(delta, __fsub_rn(wnew, wold_keep[i][j])));
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <int R, int MODE>
+__global__ void __launch_bounds__(kBlockThreads)
+asyncmesh_step_kernel(const __grid_constant__ StepParams P)
+{
+    __shared__ StageDesc sd[kMaxStages];
+    {
+        const uint32_t words = P.S * (uint32_t)(sizeof(StageDesc) / 4);
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(P.stages);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(sd);
+        for (uint32_t x = threadIdx.x; x < words; x += blockDim.x) dst[x] = src[x];
+    }
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    constexpr uint32_t wpb = kBlockThreads / 32;
+    const uint32_t n_warps = gridDim.x * wpb;
+    uint32_t s = 0;
+    for (uint32_t gc = blockIdx.x * wpb + (threadIdx.x >> 5); gc < P.total_chunks;
+         gc += n_warps) {
+        while (s + 1 < P.S && gc >= sd[s + 1].chunk_begin) ++s;
+        process_chunk<R, MODE>(P, sd[s], P.G[s], s, gc - sd[s].chunk_begin, lane);
+    }
+}
+
+}  // namespace amk

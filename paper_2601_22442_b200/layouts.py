@@ -1,0 +1,40 @@
+"""Flat parameter layouts of the benchmark workloads (host logic only).
+
+The update path sees a stage as a flat vector; only its length matters.  These
+helpers give the lengths of Llama-shaped decoder stacks split into contiguous
+pipeline stages (Section 2.1: P stages, each a contiguous run of layers).
+"""
+from __future__ import annotations
+
+from typing import Dict, List
+
+
+def llama_stage_numel(d: int, layers: int, ffn: int, vocab: int, stages: int,
+                      tied: bool) -> List[int]:
+    """Parameters per stage: per layer 4 d^2 (q, k, v, o) + 3 d ffn (gate, up,
+    down) + 2 d (two RMSNorm gains); the first stage adds the vocab x d
+    embedding, the last the final norm (d) and, if untied, the vocab x d head."""
+    if layers % stages:
+        raise ValueError("layers must divide evenly into stages")
+    per_layer = 4 * d * d + 3 * d * ffn + 2 * d
+    out = [per_layer * (layers // stages)] * stages
+    out[0] += vocab * d
+    out[-1] += d + (0 if tied else vocab * d)
+    return out
+
+
+# The benchmark configurations (R replicas, stage sizes, delay tau, steps).
+def workloads() -> Dict[str, dict]:
+    return {
+        "toy": dict(R=4, numel=[1 << 20, 1 << 20], tau=1, steps=100),
+        "llama125m": dict(R=8, numel=llama_stage_numel(768, 12, 2048, 32000, 4, True),
+                          tau=2, steps=50),
+        "llama350m": dict(R=8, numel=llama_stage_numel(1024, 24, 2816, 32000, 4, True),
+                          tau=4, steps=50),
+        "llama1b": dict(R=4, numel=llama_stage_numel(2048, 16, 5632, 32000, 8, False),
+                        tau=4, steps=20),
+    }
+
+
+DEFAULT_HP = dict(p=0.05, ema_beta=0.9, lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8,
+                  weight_decay=0.1)

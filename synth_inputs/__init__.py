@@ -78,3 +78,57 @@ def grads_host(seed: int, step: int, stage: int, R: int, coord0: int, n: int,
     return np.stack([
         normal_host(stream_key(seed, KIND_GRAD, step, stage, i), coord0, n, sigma)
         for i in range(R)])
+
+
+# ---- device fills (need the small CUDA library built from synth_fill.cu) -------
+
+import ctypes as _ct
+import os as _os
+import shutil as _sh
+import subprocess as _sp
+
+_HERE = _os.path.dirname(_os.path.abspath(__file__))
+_SRC = _os.path.join(_HERE, "synth_fill.cu")
+_LIB = _os.path.join(_HERE, "libsynth_inputs.so")
+_dev = None
+
+
+def build(force: bool = False) -> str:
+    stale = not _os.path.exists(_LIB) or _os.path.getmtime(_LIB) < _os.path.getmtime(_SRC)
+    if force or stale:
+        nvcc = _sh.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+        tmp = _LIB + ".tmp.%d" % _os.getpid()
+        _sp.run([nvcc, "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+                 "-fmad=false", "-Xcompiler", "-fPIC", "-shared", "-o", tmp, _SRC], check=True)
+        _os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _devlib():
+    global _dev
+    if _dev is None:
+        L = _ct.CDLL(build())
+        L.synth_fill_normal.restype = _ct.c_int
+        L.synth_fill_normal.argtypes = [_ct.c_void_p, _ct.c_uint64, _ct.c_uint64, _ct.c_uint64,
+                                        _ct.c_float, _ct.c_void_p]
+        _dev = L
+    return _dev
+
+
+def normal_device(dst, key: int, coord0: int, sigma: float) -> None:
+    """Fill the 1-D CUDA float32 tensor ``dst`` with the stream ``key`` starting
+    at coordinate ``coord0`` (same values as ``normal_host``)."""
+    import torch
+    assert dst.is_cuda and dst.dtype == torch.float32 and dst.is_contiguous()
+    rc = _devlib().synth_fill_normal(dst.data_ptr(), dst.numel(), coord0, key,
+                                     float(scale_f32(sigma)),
+                                     torch.cuda.current_stream(dst.device).cuda_stream)
+    if rc != 0:
+        raise RuntimeError("synth_fill_normal: CUDA error %d" % rc)
+
+
+def grads_device(dst, seed: int, step: int, stage: int, numel: int, sigma: float = 1e-3) -> None:
+    """dst: CUDA float32 [R, stride] with stride >= numel; row i <- replica i's
+    gradient of ``step``; padding columns are left untouched."""
+    for i in range(dst.shape[0]):
+        normal_device(dst[i, :numel], stream_key(seed, KIND_GRAD, step, stage, i), 0, sigma)
