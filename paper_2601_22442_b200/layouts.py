@@ -31,6 +31,8 @@ def workloads() -> Dict[str, dict]:
                           tau=2, steps=50),
         "llama350m": dict(R=8, numel=llama_stage_numel(1024, 24, 2816, 32000, 4, True),
                           tau=4, steps=50),
+        # small case for profiler captures: larger than L2, a few GB on the device
+        "profile": dict(R=4, numel=[1 << 24, 1 << 24], tau=4, steps=8),
         "llama1b": dict(R=4, numel=llama_stage_numel(2048, 16, 5632, 32000, 8, False),
                         tau=4, steps=20),
     }
