@@ -49,6 +49,10 @@ extern "C" {
 #define ASYNCMESH_FLAG_SMALL_RING 1u /* diagnostic: give each compact ring slot 1/8 of
                                         its normal capacity, so that the overflow
                                         report (DEVICE_STATUS) can be exercised    */
+#define ASYNCMESH_FLAG_DIRECT_KERNEL 2u /* use the register-load ("direct") step kernel even
+                                          where the shared-memory pipelined one applies  */
+#define ASYNCMESH_FLAG_PIPELINED_KERNEL 4u /* use the compact ring and the pipelined kernel for
+                                             any p (diagnostic: exercises its in-place path) */
 
 /* state selectors of asyncmesh_read_state */
 #define ASYNCMESH_STATE_W 0     /* weights w_i^t                               */

@@ -19,6 +19,8 @@ OK = 0
 ERR_INVALID_ARG, ERR_OOM, ERR_CUDA = -1, -2, -3
 ERR_BAD_STATE, ERR_UNSUPPORTED, ERR_DEVICE_STATUS = -4, -5, -6
 FLAG_SMALL_RING = 1
+FLAG_DIRECT_KERNEL = 2
+FLAG_PIPELINED_KERNEL = 4
 STATE = {"w": 0, "m": 1, "v": 2, "d": 3, "look": 4}
 
 ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t)

@@ -14,6 +14,7 @@
 #include <cuda_runtime.h>
 
 #include "step_kernel.cuh"
+#include "step_kernel_pipelined.cuh"
 
 using namespace amk;
 
@@ -64,6 +65,16 @@ struct DeviceScope {   // make the handle's device current for the call
 // the handle
 // ---------------------------------------------------------------------------
 
+typedef void (*step_fn)(const StepParams);
+
+constexpr int kPipeStages = 4;   // units of 2 KB in flight per warp (pipelined kernel)
+
+struct KernelChoice {
+    step_fn fn = nullptr;
+    size_t smem = 0;   // dynamic shared memory per block
+};
+
+
 struct asyncmesh {
     uint32_t R = 0, S = 0, tau = 0;
     double p = 0, ema_beta = 0, lr = 0, beta1 = 0, beta2 = 0, eps = 0, wd = 0;
@@ -86,6 +97,7 @@ struct asyncmesh {
     double *scratch = nullptr;        // one double for reductions
 
     int mode = kSync;
+    KernelChoice kernel;
     uint32_t n_slots = 0;
     uint32_t total_chunks = 0;
     int grid = 0;
@@ -214,39 +226,54 @@ static int grid_for(uint64_t items, int threads)
 // kernel dispatch
 // ---------------------------------------------------------------------------
 
-typedef void (*step_fn)(const StepParams);
-
 template <int R>
-static step_fn pick_mode(int mode)
+static KernelChoice pick_mode(int mode, bool pipelined)
 {
+    KernelChoice c;
     switch (mode) {
-    case kSync: return asyncmesh_step_kernel<R, kSync>;
-    case kCompact: return asyncmesh_step_kernel<R, kCompact>;
-    default: return asyncmesh_step_kernel<R, kDense>;
+    case kSync: c.fn = asyncmesh_step_kernel<R, kSync>; break;
+    case kDense: c.fn = asyncmesh_step_kernel<R, kDense>; break;
+    default:
+        if (pipelined) {
+            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages>;
+            c.smem = (size_t)(kBlockThreads / 32) * PipeCfg<R>::warp_bytes(kPipeStages);
+        } else {
+            c.fn = asyncmesh_step_kernel<R, kCompact>;
+        }
+    }
+    return c;
+}
+
+static KernelChoice pick_kernel(uint32_t R, int mode, bool pipelined)
+{
+    switch (R) {
+    case 1: return pick_mode<1>(mode, pipelined);
+    case 2: return pick_mode<2>(mode, pipelined);
+    case 3: return pick_mode<3>(mode, pipelined);
+    case 4: return pick_mode<4>(mode, pipelined);
+    case 5: return pick_mode<5>(mode, pipelined);
+    case 6: return pick_mode<6>(mode, pipelined);
+    case 7: return pick_mode<7>(mode, pipelined);
+    case 8: return pick_mode<8>(mode, pipelined);
+    case 9: return pick_mode<9>(mode, pipelined);
+    case 10: return pick_mode<10>(mode, pipelined);
+    case 11: return pick_mode<11>(mode, pipelined);
+    case 12: return pick_mode<12>(mode, pipelined);
+    case 13: return pick_mode<13>(mode, pipelined);
+    case 14: return pick_mode<14>(mode, pipelined);
+    case 15: return pick_mode<15>(mode, pipelined);
+    case 16: return pick_mode<16>(mode, pipelined);
+    default: return KernelChoice();
     }
 }
 
-static step_fn pick_kernel(uint32_t R, int mode)
+// The pipelined kernel stashes the selected coordinates of a sub-iteration (128
+// coordinates, union of two subsets); it pays off while they fit its stash.
+static bool stash_fits(uint32_t R, double p)
 {
-    switch (R) {
-    case 1: return pick_mode<1>(mode);
-    case 2: return pick_mode<2>(mode);
-    case 3: return pick_mode<3>(mode);
-    case 4: return pick_mode<4>(mode);
-    case 5: return pick_mode<5>(mode);
-    case 6: return pick_mode<6>(mode);
-    case 7: return pick_mode<7>(mode);
-    case 8: return pick_mode<8>(mode);
-    case 9: return pick_mode<9>(mode);
-    case 10: return pick_mode<10>(mode);
-    case 11: return pick_mode<11>(mode);
-    case 12: return pick_mode<12>(mode);
-    case 13: return pick_mode<13>(mode);
-    case 14: return pick_mode<14>(mode);
-    case 15: return pick_mode<15>(mode);
-    case 16: return pick_mode<16>(mode);
-    default: return nullptr;
-    }
+    const double q = 1.0 - (1.0 - p) * (1.0 - p);
+    const double mean = 128.0 * q, sd = std::sqrt(128.0 * q * (1.0 - q));
+    return mean + 4.0 * sd <= (R <= 4 ? 64.0 : 32.0);
 }
 
 // ---------------------------------------------------------------------------
@@ -277,7 +304,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: need lr > 0, eps > 0, weight_decay >= 0");
     if (!(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: betas must lie in [0, 1)");
-    if ((cfg->flags & ~ASYNCMESH_FLAG_SMALL_RING) != 0 || cfg->reserved != 0)
+    if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
+                        ASYNCMESH_FLAG_PIPELINED_KERNEL)) != 0 || cfg->reserved != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags, or reserved is not 0");
     if ((cfg->alloc == nullptr) != (cfg->free == nullptr))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: give both alloc and free, or neither");
@@ -345,7 +373,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
     h->total_chunks = (uint32_t)chunks;
     if (h->tau == 0) { h->mode = kSync; h->n_slots = 0; }
-    else if (dense_total <= compact_total && !(cfg->flags & ASYNCMESH_FLAG_SMALL_RING)) {
+    else if (dense_total <= compact_total &&
+             !(cfg->flags & (ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_PIPELINED_KERNEL))) {
         h->mode = kDense; h->n_slots = h->tau;
     }
     else { h->mode = kCompact; h->n_slots = h->tau + 1; }
@@ -409,12 +438,20 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
 
     // persistent grid: every SM filled to the kernel's occupancy
-    step_fn fn = pick_kernel(R, h->mode);
+    const bool pipelined = h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
+                           (stash_fits(R, cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL));
+    h->kernel = pick_kernel(R, h->mode, pipelined);
     int sms = 0, per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kBlockThreads, 0) != cudaSuccess ||
-        per_sm < 1 || sms < 1) {
-        const char *msg = cudaGetErrorString(cudaGetLastError());
+    cudaError_t ke = cudaSuccess;
+    if (h->kernel.smem > 48 * 1024)
+        ke = cudaFuncSetAttribute((const void *)h->kernel.fn,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->kernel.smem);
+    if (ke == cudaSuccess)
+        ke = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void *)h->kernel.fn,
+                                                           kBlockThreads, h->kernel.smem);
+    if (ke != cudaSuccess || per_sm < 1 || sms < 1) {
+        const char *msg = cudaGetErrorString(ke != cudaSuccess ? ke : cudaGetLastError());
         release_all(h);
         delete h;
         return fail(ASYNCMESH_ERR_CUDA, "create: the step kernel cannot run on this device: %s", msg);
@@ -527,8 +564,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
         CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
                                h->S * sizeof(unsigned int), h->stream));
 
-    step_fn fn = pick_kernel(h->R, h->mode);
-    fn<<<h->grid, kBlockThreads, 0, h->stream>>>(P);
+    h->kernel.fn<<<h->grid, kBlockThreads, h->kernel.smem, h->stream>>>(P);
     CU_TRY(cudaGetLastError());
     h->t = t;
 

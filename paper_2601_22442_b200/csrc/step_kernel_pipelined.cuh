@@ -1,0 +1,380 @@
+// Pipelined variant of the fused step for the compact snapshot ring (the
+// paper's main regime: a small subset, tau >= 1).  Same results as the direct
+// kernel of step_kernel.cuh, bit for bit; different data movement:
+//
+//  * Dense streams (w, g, m, v of one replica, 128 coordinates = one "unit" of
+//    2 KB per warp) are fetched with per-thread 16-byte asynchronous copies
+//    (cp.async) into a ring of shared-memory stages private to the warp, several
+//    units ahead of the arithmetic.  A lane reads back only what it copied, so
+//    the pipeline needs no barrier at all, only cp.async.wait_group.  The bytes
+//    in flight per SM are set by the stage count, not by registers or occupancy.
+//  * Sparse work is compacted across the warp.  The few selected coordinates of
+//    a sub-iteration (union of S^t and S^{t-tau}, ~12 of 128 at p = 0.05) are
+//    ranked with a warp scan; while the dense arithmetic runs, the owning lanes
+//    drop the values those coordinates need (w^ and w^{t-1} per replica) into a
+//    small shared-memory stash; afterwards lane q handles the q-th selected
+//    coordinate for all replicas with vector accesses to the ring and to d.
+//    Its ring and d loads are issued before the dense arithmetic starts, so
+//    their latency is hidden behind it.  Coordinates beyond the stash capacity
+//    (possible only for large p) are handled in place by their owning lane.
+#pragma once
+#include "step_kernel.cuh"
+
+namespace amk {
+
+constexpr int kUnitBytes = 4 * 32 * 16;   // w, g, m, v: one float4 per lane each
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gptr)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit()
+{
+    asm volatile("cp.async.commit_group;\n" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+template <int R>
+__device__ __forceinline__ void store_replicas(float *p, const float (&x)[R])
+{
+    if constexpr (R % 4 == 0) {
+#pragma unroll
+        for (int q = 0; q < R / 4; ++q)
+            *reinterpret_cast<float4 *>(p + 4 * q) =
+                make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]);
+    } else if constexpr (R % 2 == 0) {
+#pragma unroll
+        for (int q = 0; q < R / 2; ++q)
+            *reinterpret_cast<float2 *>(p + 2 * q) = make_float2(x[2 * q], x[2 * q + 1]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < R; ++i) p[i] = x[i];
+    }
+}
+
+template <int R>
+struct PipeCfg {
+    static constexpr int kStash = (R <= 4) ? 64 : 32;          // selected coordinates per sub-iteration
+    static constexpr int kStashWords = kStash * (2 * R + 3);   // what, wold, coord, cidx, pidx
+    static constexpr int kStashBytes = (kStashWords * 4 + 15) / 16 * 16;
+    __host__ __device__ static constexpr int warp_bytes(int stages) { return stages * kUnitBytes + kStashBytes; }
+};
+
+// Walks the warp's units in the order the arithmetic consumes them:
+// chunk (grid stride) -> sub-iteration k -> replica i.
+struct UnitCursor {
+    uint32_t gc, s, chunk;
+    int k, i, kmax;
+    bool valid;
+};
+
+__device__ __forceinline__ int sub_iterations(const StageDesc &st, uint32_t chunk)
+{
+    const uint64_t rem = st.N - (uint64_t)chunk * kWarpChunk;
+    return rem >= (uint64_t)kWarpChunk ? kSubIters : (int)((rem + 127) / 128);
+}
+
+__device__ __forceinline__ void cursor_enter_chunk(UnitCursor &c, const StageDesc *sd, uint32_t S,
+                                                   uint32_t total_chunks)
+{
+    c.valid = c.gc < total_chunks;
+    if (!c.valid) return;
+    while (c.s + 1 < S && c.gc >= sd[c.s + 1].chunk_begin) ++c.s;
+    c.chunk = c.gc - sd[c.s].chunk_begin;
+    c.kmax = sub_iterations(sd[c.s], c.chunk);
+    c.k = 0;
+    c.i = 0;
+}
+
+template <int R>
+__device__ __forceinline__ void issue_unit(const StepParams &P, const StageDesc *sd, UnitCursor &c,
+                                           uint32_t slot_addr, int lane, uint32_t n_warps)
+{
+    if (c.valid) {
+        const StageDesc &st = sd[c.s];
+        const uint64_t mu = (uint64_t)c.chunk * kWarpChunk + (uint64_t)c.k * 128 + (uint64_t)lane * 4;
+        if (mu < st.N) {
+            const uint64_t off = (uint64_t)c.i * st.stride + mu;
+            const uint32_t a = slot_addr + lane * 16;
+            cp_async16(a, st.W + off);
+            cp_async16(a + 512, P.G[c.s] + off);
+            cp_async16(a + 1024, st.M + off);
+            cp_async16(a + 1536, st.V + off);
+        }
+        if (++c.i == R) {
+            c.i = 0;
+            if (++c.k == c.kmax) {
+                c.gc += n_warps;
+                cursor_enter_chunk(c, sd, P.S, P.total_chunks);
+            }
+        }
+    }
+    cp_async_commit();   // always: keeps the group count in step with the unit count
+}
+
+template <int R, int NST>
+__global__ void __launch_bounds__(kBlockThreads)
+asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
+{
+    using Cfg = PipeCfg<R>;
+    constexpr int CAP = Cfg::kStash;
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    __shared__ StageDesc sd[kMaxStages];
+    {
+        const uint32_t words = P.S * (uint32_t)(sizeof(StageDesc) / 4);
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(P.stages);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(sd);
+        for (uint32_t x = threadIdx.x; x < words; x += blockDim.x) dst[x] = src[x];
+    }
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    constexpr uint32_t wpb = kBlockThreads / 32;
+    const uint32_t n_warps = gridDim.x * wpb;
+
+    unsigned char *my = dyn_smem + (size_t)warp * Cfg::warp_bytes(NST);
+    const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(my);
+    // stash of the current sub-iteration's selected coordinates
+    float *st_what = reinterpret_cast<float *>(my + NST * kUnitBytes);   // [CAP][R]
+    float *st_wold = st_what + CAP * R;                                  // [CAP][R]
+    uint32_t *st_coord = reinterpret_cast<uint32_t *>(st_wold + CAP * R);
+    uint32_t *st_cidx = st_coord + CAP;
+    uint32_t *st_pidx = st_cidx + CAP;
+
+    // ---- start the copy pipeline: NST - 1 units ahead --------------------------
+    UnitCursor pf;
+    pf.gc = blockIdx.x * wpb + warp;
+    pf.s = 0;
+    cursor_enter_chunk(pf, sd, P.S, P.total_chunks);
+#pragma unroll
+    for (int q = 0; q < NST - 1; ++q)
+        issue_unit<R>(P, sd, pf, stage_base + q * kUnitBytes, lane, n_warps);
+    uint32_t n = 0;   // units consumed so far
+
+    const bool consume = P.consume != 0u;
+    uint32_t s = 0;
+    for (uint32_t gc = blockIdx.x * wpb + warp; gc < P.total_chunks; gc += n_warps) {
+        while (s + 1 < P.S && gc >= sd[s + 1].chunk_begin) ++s;
+        const StageDesc &st = sd[s];
+        const uint32_t chunk = gc - st.chunk_begin;
+        const uint64_t N = st.N, stride = st.stride;
+        const uint64_t c0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
+        const int kmax = sub_iterations(st, chunk);
+
+        // ---- membership of this lane's 32 coordinates in S^t and S^{t-tau} ----
+        uint32_t pmask = 0, cmask = 0;   // bit 4k+j: coordinate c0 + 128k + j
+#pragma unroll 2
+        for (int k = 0; k < kSubIters; ++k) {
+            const uint64_t mu = c0 + (uint64_t)k * 128;
+            if (mu < N) {
+                const uint64_t left = N - mu;
+                const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
+                const uint32_t quad = (uint32_t)(mu >> 2);
+                pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * k);
+                if (consume)
+                    cmask |= (subset_bits(P.rule, st.stage_id, P.cons_step, quad) & valid) << (4 * k);
+            }
+        }
+
+        // ---- room in the producing slot, position in the consumed slot ---------
+        uint32_t pbase = 0, cbase = 0, cexcl = 0, total;
+        const uint32_t pexcl = warp_exclusive_sum(__popc(pmask), lane, total);
+        if (lane == 0) {
+            uint32_t b = 0;
+            if (total) {
+                b = atomicAdd(&P.cursors[P.prod_slot * P.S + s], total);
+                if (b > st.cap || total > st.cap - b) {   // slot full: drop loudly
+                    b = kInvalidBase;
+                    atomicExch(P.status, kStatusRingOverflow);
+                }
+            }
+            st.chunk_base[(uint64_t)P.prod_slot * st.n_chunks + chunk] = b;
+            pbase = b;
+        }
+        pbase = __shfl_sync(kFullMask, pbase, 0);
+        if (pbase == kInvalidBase) pmask = 0;
+        if (consume) {
+            cbase = st.chunk_base[(uint64_t)P.cons_slot * st.n_chunks + chunk];
+            if (cbase == kInvalidBase) cmask = 0;
+            uint32_t ctotal;
+            cexcl = warp_exclusive_sum(__popc(cmask), lane, ctotal);
+        }
+        const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
+        float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
+        const float delta = st.delta;
+        const bool has_look = st.has_look != 0u;
+
+#pragma unroll 1
+        for (int k = 0; k < kmax; ++k) {
+            const uint64_t mu = c0 + (uint64_t)k * 128;
+            const bool active = mu < N;
+            const uint32_t pm = (pmask >> (4 * k)) & 0xFu;
+            const uint32_t cm = (cmask >> (4 * k)) & 0xFu;
+            const uint32_t um = pm | cm;
+
+            // ---- rank the selected coordinates of this sub-iteration ------------
+            uint32_t n_u;
+            const uint32_t uexcl = warp_exclusive_sum(__popc(um), lane, n_u);
+            const uint32_t cfirst = cbase + cexcl + __popc(cmask & ((1u << (4 * k)) - 1u));
+            const uint32_t pfirst = pbase + pexcl + __popc(pmask & ((1u << (4 * k)) - 1u));
+            uint32_t sm = 0;   // bits of um that fit the stash
+            if (um) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if ((um >> j) & 1u) {
+                        const uint32_t below = (1u << j) - 1u;
+                        const uint32_t r = uexcl + __popc(um & below);
+                        if (r < (uint32_t)CAP) {
+                            sm |= 1u << j;
+                            st_coord[r] = (uint32_t)(mu + j);
+                            st_cidx[r] = ((cm >> j) & 1u) ? cfirst + __popc(cm & below) : kInvalidBase;
+                            st_pidx[r] = ((pm >> j) & 1u) ? pfirst + __popc(pm & below) : kInvalidBase;
+                        }
+                    }
+                }
+            }
+            const uint32_t om = um & ~sm;   // handled in place (only when the stash is full)
+            __syncwarp();
+
+            // ---- lane q adopts the q-th selected coordinate; its loads go out now
+            const uint32_t n_s = n_u < (uint32_t)CAP ? n_u : (uint32_t)CAP;
+            uint32_t e_coord = 0, e_c = kInvalidBase, e_p = kInvalidBase;
+            float s_old[R], s_dd[R];
+#pragma unroll
+            for (int i = 0; i < R; ++i) { s_old[i] = 0.f; s_dd[i] = 0.f; }
+            if ((uint32_t)lane < n_s) {
+                e_coord = st_coord[lane];
+                e_c = st_cidx[lane];
+                e_p = st_pidx[lane];
+                if (e_c != kInvalidBase) {
+                    load_replicas<R>(ring_cons + (uint64_t)e_c * R, s_old);
+                    load_replicas<R>(st.D + (uint64_t)e_coord * R, s_dd);
+                }
+            }
+
+            // ---- dense arithmetic, one replica (= one pipeline unit) at a time ----
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                cp_async_wait<NST - 2>();
+                issue_unit<R>(P, sd, pf, stage_base + ((n + NST - 1) % NST) * kUnitBytes, lane, n_warps);
+                const unsigned char *slot = my + (n % NST) * kUnitBytes + lane * 16;
+                ++n;
+                if (active) {
+                    const float4 w4 = *reinterpret_cast<const float4 *>(slot);
+                    const float4 g4 = *reinterpret_cast<const float4 *>(slot + 512);
+                    const float4 m4 = *reinterpret_cast<const float4 *>(slot + 1024);
+                    const float4 v4 = *reinterpret_cast<const float4 *>(slot + 1536);
+                    const uint64_t off = (uint64_t)i * stride + mu;
+                    const float w[4] = {w4.x, w4.y, w4.z, w4.w};
+                    const float g[4] = {g4.x, g4.y, g4.z, g4.w};
+                    float m[4] = {m4.x, m4.y, m4.z, m4.w};
+                    float v[4] = {v4.x, v4.y, v4.z, v4.w};
+                    float wh[4], wn[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        adamw(P, w[c], g[c], m[c], v[c], wh[c]);
+                        wn[c] = wh[c];
+                    }
+                    st_stream(st.M + off, m);
+                    st_stream(st.V + off, v);
+
+                    if (sm) {   // hand w^ and w^{t-1} of selected coordinates to the stash
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if ((sm >> j) & 1u) {
+                                const uint32_t r = uexcl + __popc(um & ((1u << j) - 1u));
+                                st_what[r * R + i] = wh[j];
+                                st_wold[r * R + i] = w[j];
+                            }
+                        }
+                    }
+                    if (om) {   // stash full: this lane does the sparse work itself
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if ((om >> j) & 1u) {
+                                const uint32_t below = (1u << j) - 1u;
+                                if ((cm >> j) & 1u) {
+                                    const uint64_t ce = (uint64_t)(cfirst + __popc(cm & below)) * R;
+                                    float old[R];
+                                    load_replicas<R>(ring_cons + ce, old);
+                                    float a = old[0];
+#pragma unroll
+                                    for (int q = 1; q < R; ++q) a = __fadd_rn(a, old[q]);
+                                    const float abar = __fdiv_rn(a, P.Rf);
+                                    float *dp = st.D + (mu + j) * R + i;
+                                    const float diff = __fsub_rn(wh[j], old[i]);
+                                    const float dn = __fadd_rn(__fmul_rn(P.oml, *dp), __fmul_rn(P.lam, diff));
+                                    *dp = dn;
+                                    wn[j] = __fadd_rn(abar, dn);
+                                }
+                                if ((pm >> j) & 1u)
+                                    ring_prod[(uint64_t)(pfirst + __popc(pm & below)) * R + i] = wh[j];
+                            }
+                        }
+                    }
+
+                    st_stream(st.W + off, wn);
+                    if (has_look) {   // Section 2.2: extrapolate the last update direction
+                        float lk[4];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            lk[c] = __fadd_rn(wn[c], __fmul_rn(delta, __fsub_rn(wn[c], w[c])));
+                        st_stream(st.LOOK + off, lk);
+                    }
+                }
+            }
+            __syncwarp();   // stash complete; dense stores ordered before the fix-ups below
+
+            // ---- sparse phase: lane q finishes the q-th selected coordinate -------
+            for (uint32_t r0 = 0; r0 < n_s; r0 += 32) {
+                const uint32_t q = r0 + lane;
+                if (q < n_s) {
+                    if (r0 != 0) {   // second round (stash of 64): loads were not issued ahead
+                        e_coord = st_coord[q];
+                        e_c = st_cidx[q];
+                        e_p = st_pidx[q];
+                        if (e_c != kInvalidBase) {
+                            load_replicas<R>(ring_cons + (uint64_t)e_c * R, s_old);
+                            load_replicas<R>(st.D + (uint64_t)e_coord * R, s_dd);
+                        }
+                    }
+                    float wh[R];
+                    load_replicas<R>(st_what + q * R, wh);
+                    if (e_c != kInvalidBase) {
+                        // Eq. "ema" + corrected averaging on S^{t-tau}
+                        float wold[R];
+                        load_replicas<R>(st_wold + q * R, wold);
+                        float a = s_old[0];
+#pragma unroll
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, s_old[i]);
+                        const float abar = __fdiv_rn(a, P.Rf);
+#pragma unroll
+                        for (int i = 0; i < R; ++i) {
+                            const float diff = __fsub_rn(wh[i], s_old[i]);
+                            const float dn = __fadd_rn(__fmul_rn(P.oml, s_dd[i]), __fmul_rn(P.lam, diff));
+                            s_dd[i] = dn;
+                            const float wnew = __fadd_rn(abar, dn);
+                            const uint64_t o1 = (uint64_t)i * stride + e_coord;
+                            st.W[o1] = wnew;
+                            if (has_look)
+                                st.LOOK[o1] = __fadd_rn(wnew, __fmul_rn(delta, __fsub_rn(wnew, wold[i])));
+                        }
+                        store_replicas<R>(st.D + (uint64_t)e_coord * R, s_dd);
+                    }
+                    if (e_p != kInvalidBase)   // snapshot of the local iterate on S^t
+                        store_replicas<R>(ring_prod + (uint64_t)e_p * R, wh);
+                }
+            }
+            __syncwarp();   // the stash may be overwritten by the next sub-iteration
+        }
+    }
+    cp_async_wait<0>();
+}
+
+}  // namespace amk

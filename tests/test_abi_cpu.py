@@ -63,7 +63,7 @@ def _cfg(**over):
     (dict(R=0), "R ="), (dict(R=17), "R ="), (dict(S=0), "S ="), (dict(S=65), "S ="),
     (dict(p=-0.1), "p ="), (dict(p=1.5), "p ="), (dict(p=float("nan")), "p ="),
     (dict(tau=65), "tau"), (dict(ema_beta=1.01), "ema_beta"), (dict(lr=0.0), "lr"),
-    (dict(eps=0.0), "eps"), (dict(beta1=1.0), "betas"), (dict(flags=2), "flags"),
+    (dict(eps=0.0), "eps"), (dict(beta1=1.0), "betas"), (dict(flags=8), "flags"),
 ])
 def test_create_rejects_bad_arguments_without_touching_a_device(lib, over, word):
     h = ctypes.c_void_p()

@@ -26,11 +26,11 @@ def am():
 
 
 def make_pair(R, numel, p, tau, lam, delays=None, seed=0x5EED, hp=HP, same_init=True,
-              init_seed=0x1217):
+              init_seed=0x1217, flags=0):
     o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
                       lookahead_delay=delays, **hp)
     g = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
-                       lookahead_delay=delays, **hp)
+                       lookahead_delay=delays, flags=flags, **hp)
     for s, n in enumerate(numel):
         if same_init:
             w0 = si.init_weights_host(init_seed, s, 0, n)
@@ -140,7 +140,19 @@ def test_modes_small(tau, p):
 @pytest.mark.parametrize("R", [1, 2, 3, 5, 7, 8, 12, 16])
 def test_replica_counts(R):
     run_case(R, [2500], 0.3, 2, 0.9, steps=7)
+    run_case(R, [2500], 0.05, 2, 0.9, steps=7)
     run_case(R, [2500], 0.3, 0, 0.9, steps=3)
+
+
+@pytest.mark.parametrize("flag", ["direct", "pipelined"])
+@pytest.mark.parametrize("R,p", [(4, 0.05), (8, 0.05), (3, 0.1), (4, 0.5), (8, 0.35), (2, 1.0), (5, 0.9)])
+def test_both_compact_ring_kernels(flag, R, p):
+    # the register-load kernel and the shared-memory pipelined kernel are two routes
+    # to the same numbers; large p forces the pipelined kernel through its in-place
+    # path (more selected coordinates per sub-iteration than its stash holds)
+    from paper_2601_22442_b200 import binding
+    f = binding.FLAG_DIRECT_KERNEL if flag == "direct" else binding.FLAG_PIPELINED_KERNEL
+    run_case(R, [9000, 1024 * 3 + 5, 77], p, 2, 0.9, steps=7, flags=f)
 
 
 def test_ragged_stage_sizes():
