@@ -67,11 +67,11 @@ struct DeviceScope {   // make the handle's device current for the call
 
 typedef void (*step_fn)(const StepParams);
 
-constexpr int kPipeStages = 4;   // units of 2 KB in flight per warp (pipelined kernel)
 
 struct KernelChoice {
     step_fn fn = nullptr;
-    size_t smem = 0;   // dynamic shared memory per block
+    size_t smem = 0;              // dynamic shared memory per block
+    int threads = kBlockThreads;  // block size
 };
 
 
@@ -227,7 +227,7 @@ static int grid_for(uint64_t items, int threads)
 // ---------------------------------------------------------------------------
 
 template <int R>
-static KernelChoice pick_mode(int mode, bool pipelined)
+static KernelChoice pick_mode(int mode, bool pipelined, uint32_t S)
 {
     KernelChoice c;
     switch (mode) {
@@ -235,8 +235,10 @@ static KernelChoice pick_mode(int mode, bool pipelined)
     case kDense: c.fn = asyncmesh_step_kernel<R, kDense>; break;
     default:
         if (pipelined) {
-            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages>;
-            c.smem = (size_t)(kBlockThreads / 32) * PipeCfg<R>::warp_bytes(kPipeStages);
+            c.fn = asyncmesh_step_kernel_pipelined<R, AM_PIPE_STAGES>;
+            c.threads = kPipeThreads;
+            c.smem = (size_t)pipe_table_bytes(S) +
+                     (size_t)(kPipeThreads / 32) * PipeCfg<R>::warp_bytes(AM_PIPE_STAGES);
         } else {
             c.fn = asyncmesh_step_kernel<R, kCompact>;
         }
@@ -244,36 +246,36 @@ static KernelChoice pick_mode(int mode, bool pipelined)
     return c;
 }
 
-static KernelChoice pick_kernel(uint32_t R, int mode, bool pipelined)
+static KernelChoice pick_kernel(uint32_t R, int mode, bool pipelined, uint32_t S)
 {
     switch (R) {
-    case 1: return pick_mode<1>(mode, pipelined);
-    case 2: return pick_mode<2>(mode, pipelined);
-    case 3: return pick_mode<3>(mode, pipelined);
-    case 4: return pick_mode<4>(mode, pipelined);
-    case 5: return pick_mode<5>(mode, pipelined);
-    case 6: return pick_mode<6>(mode, pipelined);
-    case 7: return pick_mode<7>(mode, pipelined);
-    case 8: return pick_mode<8>(mode, pipelined);
-    case 9: return pick_mode<9>(mode, pipelined);
-    case 10: return pick_mode<10>(mode, pipelined);
-    case 11: return pick_mode<11>(mode, pipelined);
-    case 12: return pick_mode<12>(mode, pipelined);
-    case 13: return pick_mode<13>(mode, pipelined);
-    case 14: return pick_mode<14>(mode, pipelined);
-    case 15: return pick_mode<15>(mode, pipelined);
-    case 16: return pick_mode<16>(mode, pipelined);
+    case 1: return pick_mode<1>(mode, pipelined, S);
+    case 2: return pick_mode<2>(mode, pipelined, S);
+    case 3: return pick_mode<3>(mode, pipelined, S);
+    case 4: return pick_mode<4>(mode, pipelined, S);
+    case 5: return pick_mode<5>(mode, pipelined, S);
+    case 6: return pick_mode<6>(mode, pipelined, S);
+    case 7: return pick_mode<7>(mode, pipelined, S);
+    case 8: return pick_mode<8>(mode, pipelined, S);
+    case 9: return pick_mode<9>(mode, pipelined, S);
+    case 10: return pick_mode<10>(mode, pipelined, S);
+    case 11: return pick_mode<11>(mode, pipelined, S);
+    case 12: return pick_mode<12>(mode, pipelined, S);
+    case 13: return pick_mode<13>(mode, pipelined, S);
+    case 14: return pick_mode<14>(mode, pipelined, S);
+    case 15: return pick_mode<15>(mode, pipelined, S);
+    case 16: return pick_mode<16>(mode, pipelined, S);
     default: return KernelChoice();
     }
 }
 
-// The pipelined kernel stashes the selected coordinates of a sub-iteration (128
-// coordinates, union of two subsets); it pays off while they fit its stash.
-static bool stash_fits(uint32_t R, double p)
+// The pipelined kernel stashes the selected coordinates of a sub-iteration
+// (union of two subsets); it pays off while they fit its stash.
+static bool stash_fits(double p)
 {
     const double q = 1.0 - (1.0 - p) * (1.0 - p);
-    const double mean = 128.0 * q, sd = std::sqrt(128.0 * q * (1.0 - q));
-    return mean + 4.0 * sd <= (R <= 4 ? 64.0 : 32.0);
+    const double mean = kPipeSubCoords * q, sd = std::sqrt(kPipeSubCoords * q * (1.0 - q));
+    return mean + 4.0 * sd <= (double)PipeCfg<4>::kStash;
 }
 
 // ---------------------------------------------------------------------------
@@ -439,8 +441,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
 
     // persistent grid: every SM filled to the kernel's occupancy
     const bool pipelined = h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
-                           (stash_fits(R, cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL));
-    h->kernel = pick_kernel(R, h->mode, pipelined);
+                           (stash_fits(cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL));
+    h->kernel = pick_kernel(R, h->mode, pipelined, S);
     int sms = 0, per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
     cudaError_t ke = cudaSuccess;
@@ -449,7 +451,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->kernel.smem);
     if (ke == cudaSuccess)
         ke = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void *)h->kernel.fn,
-                                                           kBlockThreads, h->kernel.smem);
+                                                           h->kernel.threads, h->kernel.smem);
     if (ke != cudaSuccess || per_sm < 1 || sms < 1) {
         const char *msg = cudaGetErrorString(ke != cudaSuccess ? ke : cudaGetLastError());
         release_all(h);
@@ -457,7 +459,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         return fail(ASYNCMESH_ERR_CUDA, "create: the step kernel cannot run on this device: %s", msg);
     }
     uint64_t blocks = (uint64_t)sms * per_sm;
-    const uint64_t need = ((uint64_t)h->total_chunks + kBlockThreads / 32 - 1) / (kBlockThreads / 32);
+    const uint64_t wpb = (uint64_t)h->kernel.threads / 32;
+    const uint64_t need = ((uint64_t)h->total_chunks + wpb - 1) / wpb;
     if (blocks > need) blocks = need;
     h->grid = (int)blocks;
 
@@ -564,7 +567,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
         CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
                                h->S * sizeof(unsigned int), h->stream));
 
-    h->kernel.fn<<<h->grid, kBlockThreads, h->kernel.smem, h->stream>>>(P);
+    h->kernel.fn<<<h->grid, h->kernel.threads, h->kernel.smem, h->stream>>>(P);
     CU_TRY(cudaGetLastError());
     h->t = t;
 
@@ -791,3 +794,4 @@ extern "C" int asyncmesh_debug_philox(int device, const uint32_t *ctr_host, cons
     if (e != cudaSuccess) return fail(ASYNCMESH_ERR_CUDA, "debug_philox: %s", cudaGetErrorString(e));
     return ASYNCMESH_OK;
 }
+

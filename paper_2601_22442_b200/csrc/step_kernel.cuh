@@ -94,8 +94,13 @@ __device__ __forceinline__ void adamw(const StepParams &P, float w, float g, flo
     v = __fadd_rn(__fmul_rn(P.b2, v), __fmul_rn(P.omb2, __fmul_rn(g, g)));
     const float mh = __fmul_rn(m, P.ib1);
     const float vh = __fmul_rn(v, P.ib2);
+#ifdef AM_EXPERIMENT_FAST_MATH   // timing experiment only: not IEEE, breaks parity
+    const float den = __fadd_rn(__fmul_rn(vh, rsqrtf(vh)), P.eps);
+    const float u = __fdividef(mh, den);
+#else
     const float den = __fadd_rn(__fsqrt_rn(vh), P.eps);
     const float u = __fdiv_rn(mh, den);
+#endif
     const float decayed = __fsub_rn(w, __fmul_rn(P.lrwd, w));
     what = __fsub_rn(decayed, __fmul_rn(P.lr, u));
 }

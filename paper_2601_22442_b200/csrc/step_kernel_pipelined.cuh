@@ -2,27 +2,53 @@
 // paper's main regime: a small subset, tau >= 1).  Same results as the direct
 // kernel of step_kernel.cuh, bit for bit; different data movement:
 //
-//  * Dense streams (w, g, m, v of one replica, 128 coordinates = one "unit" of
-//    2 KB per warp) are fetched with per-thread 16-byte asynchronous copies
-//    (cp.async) into a ring of shared-memory stages private to the warp, several
-//    units ahead of the arithmetic.  A lane reads back only what it copied, so
-//    the pipeline needs no barrier at all, only cp.async.wait_group.  The bytes
-//    in flight per SM are set by the stage count, not by registers or occupancy.
-//  * Sparse work is compacted across the warp.  The few selected coordinates of
-//    a sub-iteration (union of S^t and S^{t-tau}, ~12 of 128 at p = 0.05) are
+//  * Dense streams.  A warp walks its chunk in sub-iterations of V x 128
+//    coordinates; per sub-iteration and replica it needs w, g, m, v as V float4
+//    per lane and array (one "unit", V x 2 KB).  Units are fetched with
+//    per-thread 16-byte asynchronous copies (cp.async) into a ring of shared-
+//    memory stages private to the warp, ahead of the arithmetic.  A lane reads
+//    back only what it copied itself, so the pipeline needs no barrier, only
+//    cp.async.wait_group; the bytes in flight per SM are set by the stage count,
+//    not by registers or occupancy.  With V = 2 a lane carries eight independent
+//    coordinates through the optimizer arithmetic, which is what keeps the issue
+//    slots busy between the long IEEE divide / square-root sequences.
+//  * Sparse work is compacted across the warp.  The selected coordinates of a
+//    sub-iteration (union of S^t and S^{t-tau}, ~25 of 256 at p = 0.05) are
 //    ranked with a warp scan; while the dense arithmetic runs, the owning lanes
 //    drop the values those coordinates need (w^ and w^{t-1} per replica) into a
-//    small shared-memory stash; afterwards lane q handles the q-th selected
+//    small shared-memory stash; afterwards lane q finishes the q-th selected
 //    coordinate for all replicas with vector accesses to the ring and to d.
 //    Its ring and d loads are issued before the dense arithmetic starts, so
-//    their latency is hidden behind it.  Coordinates beyond the stash capacity
+//    their latency hides behind it.  Coordinates beyond the stash capacity
 //    (possible only for large p) are handled in place by their owning lane.
 #pragma once
 #include "step_kernel.cuh"
 
+#ifndef AM_PIPE_STAGES
+#define AM_PIPE_STAGES 3      // units in the shared-memory ring of a warp
+#endif
+#ifndef AM_PIPE_MIN_BLOCKS
+#define AM_PIPE_MIN_BLOCKS 2  // blocks per SM the register budget is sized for
+#endif
+#ifndef AM_PIPE_WIDTH
+#define AM_PIPE_WIDTH 2       // float4 per lane, array and unit (V)
+#endif
+#ifndef AM_PIPE_STASH
+#define AM_PIPE_STASH 64      // selected coordinates a sub-iteration can stash
+#endif
+#ifndef AM_PIPE_THREADS
+#define AM_PIPE_THREADS 192
+#endif
+
 namespace amk {
 
-constexpr int kUnitBytes = 4 * 32 * 16;   // w, g, m, v: one float4 per lane each
+constexpr int kPipeV = AM_PIPE_WIDTH;
+constexpr int kPipeThreads = AM_PIPE_THREADS;
+constexpr int kPipeSubCoords = 128 * kPipeV;            // coordinates per sub-iteration
+constexpr int kPipeSubIters = kWarpChunk / kPipeSubCoords;
+constexpr int kPipeBits = 4 * kPipeV;                   // mask bits per lane and sub-iteration
+constexpr int kUnitBytes = 4 * kPipeV * 512;            // w, g, m, v: V float4 per lane each
+static_assert(kPipeSubIters * kPipeBits == 32, "a lane's chunk mask must fill 32 bits");
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr)
 {
@@ -59,58 +85,79 @@ __device__ __forceinline__ void store_replicas(float *p, const float (&x)[R])
 
 template <int R>
 struct PipeCfg {
-    static constexpr int kStash = (R <= 4) ? 64 : 32;          // selected coordinates per sub-iteration
+    static constexpr int kStash = AM_PIPE_STASH;
     static constexpr int kStashWords = kStash * (2 * R + 3);   // what, wold, coord, cidx, pidx
     static constexpr int kStashBytes = (kStashWords * 4 + 15) / 16 * 16;
-    __host__ __device__ static constexpr int warp_bytes(int stages) { return stages * kUnitBytes + kStashBytes; }
+    __host__ __device__ static constexpr int warp_bytes(int stages)
+    {
+        return stages * kUnitBytes + kStashBytes;
+    }
 };
 
-// Walks the warp's units in the order the arithmetic consumes them:
-// chunk (grid stride) -> sub-iteration k -> replica i.
+// Dynamic shared memory: the stage table (S entries), then one region per warp.
+__host__ __device__ constexpr int pipe_table_bytes(uint32_t S)
+{
+    return (int)((S * sizeof(StageDesc) + 15) / 16 * 16);
+}
+
+__device__ __forceinline__ int pipe_sub_iterations(uint64_t N, uint32_t chunk)
+{
+    const uint64_t rem = N - (uint64_t)chunk * kWarpChunk;
+    return rem >= (uint64_t)kWarpChunk ? kPipeSubIters
+                                       : (int)((rem + kPipeSubCoords - 1) / kPipeSubCoords);
+}
+
+// Walks the warp's units in the order the arithmetic consumes them (chunk by
+// grid stride -> sub-iteration k -> replica i) and issues their copies.  The
+// stage's pointers live in registers and are refreshed when the chunk changes.
 struct UnitCursor {
-    uint32_t gc, s, chunk;
+    const float *W, *G, *M, *V;   // of the current stage
+    uint64_t N, stride;
+    uint64_t mu0;                 // first coordinate of this lane in the current sub-iteration
+    uint32_t gc, s;
     int k, i, kmax;
     bool valid;
 };
 
-__device__ __forceinline__ int sub_iterations(const StageDesc &st, uint32_t chunk)
+__device__ __forceinline__ void cursor_enter_chunk(UnitCursor &c, const StepParams &P,
+                                                   const StageDesc *sd, int lane)
 {
-    const uint64_t rem = st.N - (uint64_t)chunk * kWarpChunk;
-    return rem >= (uint64_t)kWarpChunk ? kSubIters : (int)((rem + 127) / 128);
-}
-
-__device__ __forceinline__ void cursor_enter_chunk(UnitCursor &c, const StageDesc *sd, uint32_t S,
-                                                   uint32_t total_chunks)
-{
-    c.valid = c.gc < total_chunks;
+    c.valid = c.gc < P.total_chunks;
     if (!c.valid) return;
-    while (c.s + 1 < S && c.gc >= sd[c.s + 1].chunk_begin) ++c.s;
-    c.chunk = c.gc - sd[c.s].chunk_begin;
-    c.kmax = sub_iterations(sd[c.s], c.chunk);
+    while (c.s + 1 < P.S && c.gc >= sd[c.s + 1].chunk_begin) ++c.s;
+    const StageDesc &st = sd[c.s];
+    const uint32_t chunk = c.gc - st.chunk_begin;
+    c.W = st.W; c.M = st.M; c.V = st.V; c.G = P.G[c.s];
+    c.N = st.N; c.stride = st.stride;
+    c.kmax = pipe_sub_iterations(st.N, chunk);
     c.k = 0;
     c.i = 0;
+    c.mu0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
 }
 
 template <int R>
-__device__ __forceinline__ void issue_unit(const StepParams &P, const StageDesc *sd, UnitCursor &c,
+__device__ __forceinline__ void issue_unit(UnitCursor &c, const StepParams &P, const StageDesc *sd,
                                            uint32_t slot_addr, int lane, uint32_t n_warps)
 {
     if (c.valid) {
-        const StageDesc &st = sd[c.s];
-        const uint64_t mu = (uint64_t)c.chunk * kWarpChunk + (uint64_t)c.k * 128 + (uint64_t)lane * 4;
-        if (mu < st.N) {
-            const uint64_t off = (uint64_t)c.i * st.stride + mu;
-            const uint32_t a = slot_addr + lane * 16;
-            cp_async16(a, st.W + off);
-            cp_async16(a + 512, P.G[c.s] + off);
-            cp_async16(a + 1024, st.M + off);
-            cp_async16(a + 1536, st.V + off);
+        const uint32_t a = slot_addr + lane * 16;
+#pragma unroll
+        for (int h = 0; h < kPipeV; ++h) {
+            const uint64_t mu = c.mu0 + (uint64_t)h * 128;
+            if (mu < c.N) {
+                const uint64_t off = (uint64_t)c.i * c.stride + mu;
+                cp_async16(a + (0 * kPipeV + h) * 512, c.W + off);
+                cp_async16(a + (1 * kPipeV + h) * 512, c.G + off);
+                cp_async16(a + (2 * kPipeV + h) * 512, c.M + off);
+                cp_async16(a + (3 * kPipeV + h) * 512, c.V + off);
+            }
         }
         if (++c.i == R) {
             c.i = 0;
+            c.mu0 += kPipeSubCoords;
             if (++c.k == c.kmax) {
                 c.gc += n_warps;
-                cursor_enter_chunk(c, sd, P.S, P.total_chunks);
+                cursor_enter_chunk(c, P, sd, lane);
             }
         }
     }
@@ -118,13 +165,16 @@ __device__ __forceinline__ void issue_unit(const StepParams &P, const StageDesc 
 }
 
 template <int R, int NST>
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kPipeThreads, AM_PIPE_MIN_BLOCKS)
 asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 {
     using Cfg = PipeCfg<R>;
     constexpr int CAP = Cfg::kStash;
-    extern __shared__ __align__(16) unsigned char dyn_smem[];
-    __shared__ StageDesc sd[kMaxStages];
+    constexpr int V = kPipeV;
+    constexpr int NB = kPipeBits;   // mask bits per lane and sub-iteration
+    extern __shared__ __align__(16) unsigned char dyn_smem_all[];
+    StageDesc *sd = reinterpret_cast<StageDesc *>(dyn_smem_all);
+    unsigned char *dyn_smem = dyn_smem_all + pipe_table_bytes(P.S);
     {
         const uint32_t words = P.S * (uint32_t)(sizeof(StageDesc) / 4);
         const uint32_t *src = reinterpret_cast<const uint32_t *>(P.stages);
@@ -135,7 +185,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    constexpr uint32_t wpb = kBlockThreads / 32;
+    constexpr uint32_t wpb = kPipeThreads / 32;
     const uint32_t n_warps = gridDim.x * wpb;
 
     unsigned char *my = dyn_smem + (size_t)warp * Cfg::warp_bytes(NST);
@@ -151,10 +201,10 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
     UnitCursor pf;
     pf.gc = blockIdx.x * wpb + warp;
     pf.s = 0;
-    cursor_enter_chunk(pf, sd, P.S, P.total_chunks);
+    cursor_enter_chunk(pf, P, sd, lane);
 #pragma unroll
     for (int q = 0; q < NST - 1; ++q)
-        issue_unit<R>(P, sd, pf, stage_base + q * kUnitBytes, lane, n_warps);
+        issue_unit<R>(pf, P, sd, stage_base + q * kUnitBytes, lane, n_warps);
     uint32_t n = 0;   // units consumed so far
 
     const bool consume = P.consume != 0u;
@@ -165,25 +215,30 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         const uint32_t chunk = gc - st.chunk_begin;
         const uint64_t N = st.N, stride = st.stride;
         const uint64_t c0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
-        const int kmax = sub_iterations(st, chunk);
+        const int kmax = pipe_sub_iterations(N, chunk);
+
+        // position of this chunk in the consumed slot: ask early, use late
+        uint32_t cbase = 0;
+        if (consume) cbase = st.chunk_base[(uint64_t)P.cons_slot * st.n_chunks + chunk];
 
         // ---- membership of this lane's 32 coordinates in S^t and S^{t-tau} ----
-        uint32_t pmask = 0, cmask = 0;   // bit 4k+j: coordinate c0 + 128k + j
+        // bit 4b + c  <->  coordinate c0 + 128 b + c; sub-iteration k owns bits NB*k ..
+        uint32_t pmask = 0, cmask = 0;
 #pragma unroll 2
-        for (int k = 0; k < kSubIters; ++k) {
-            const uint64_t mu = c0 + (uint64_t)k * 128;
+        for (int b = 0; b < 8; ++b) {   // 8 quads per lane and chunk
+            const uint64_t mu = c0 + (uint64_t)b * 128;
             if (mu < N) {
                 const uint64_t left = N - mu;
                 const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
                 const uint32_t quad = (uint32_t)(mu >> 2);
-                pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * k);
+                pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * b);
                 if (consume)
-                    cmask |= (subset_bits(P.rule, st.stage_id, P.cons_step, quad) & valid) << (4 * k);
+                    cmask |= (subset_bits(P.rule, st.stage_id, P.cons_step, quad) & valid) << (4 * b);
             }
         }
 
-        // ---- room in the producing slot, position in the consumed slot ---------
-        uint32_t pbase = 0, cbase = 0, cexcl = 0, total;
+        // ---- room in the producing slot -----------------------------------------
+        uint32_t pbase = 0, cexcl = 0, total;
         const uint32_t pexcl = warp_exclusive_sum(__popc(pmask), lane, total);
         if (lane == 0) {
             uint32_t b = 0;
@@ -197,14 +252,13 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
             st.chunk_base[(uint64_t)P.prod_slot * st.n_chunks + chunk] = b;
             pbase = b;
         }
-        pbase = __shfl_sync(kFullMask, pbase, 0);
-        if (pbase == kInvalidBase) pmask = 0;
         if (consume) {
-            cbase = st.chunk_base[(uint64_t)P.cons_slot * st.n_chunks + chunk];
             if (cbase == kInvalidBase) cmask = 0;
             uint32_t ctotal;
             cexcl = warp_exclusive_sum(__popc(cmask), lane, ctotal);
         }
+        pbase = __shfl_sync(kFullMask, pbase, 0);
+        if (pbase == kInvalidBase) pmask = 0;
         const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
         float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
         const float delta = st.delta;
@@ -212,27 +266,28 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 
 #pragma unroll 1
         for (int k = 0; k < kmax; ++k) {
-            const uint64_t mu = c0 + (uint64_t)k * 128;
-            const bool active = mu < N;
-            const uint32_t pm = (pmask >> (4 * k)) & 0xFu;
-            const uint32_t cm = (cmask >> (4 * k)) & 0xFu;
+            const uint64_t mu0 = c0 + (uint64_t)k * kPipeSubCoords;   // h = 0; h adds 128
+            constexpr uint32_t kSubMask = (NB == 32) ? 0xFFFFFFFFu : ((1u << (NB % 32)) - 1u);
+            const uint32_t lowbits = (k == 0) ? 0u : ((1u << ((NB * k) % 32)) - 1u);
+            const uint32_t pm = (pmask >> (NB * k)) & kSubMask;
+            const uint32_t cm = (cmask >> (NB * k)) & kSubMask;
             const uint32_t um = pm | cm;
 
             // ---- rank the selected coordinates of this sub-iteration ------------
             uint32_t n_u;
             const uint32_t uexcl = warp_exclusive_sum(__popc(um), lane, n_u);
-            const uint32_t cfirst = cbase + cexcl + __popc(cmask & ((1u << (4 * k)) - 1u));
-            const uint32_t pfirst = pbase + pexcl + __popc(pmask & ((1u << (4 * k)) - 1u));
+            const uint32_t cfirst = cbase + cexcl + __popc(cmask & lowbits);
+            const uint32_t pfirst = pbase + pexcl + __popc(pmask & lowbits);
             uint32_t sm = 0;   // bits of um that fit the stash
             if (um) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < NB; ++j) {
                     if ((um >> j) & 1u) {
                         const uint32_t below = (1u << j) - 1u;
                         const uint32_t r = uexcl + __popc(um & below);
                         if (r < (uint32_t)CAP) {
                             sm |= 1u << j;
-                            st_coord[r] = (uint32_t)(mu + j);
+                            st_coord[r] = (uint32_t)(mu0 + (uint64_t)(j >> 2) * 128 + (j & 3));
                             st_cidx[r] = ((cm >> j) & 1u) ? cfirst + __popc(cm & below) : kInvalidBase;
                             st_pidx[r] = ((pm >> j) & 1u) ? pfirst + __popc(pm & below) : kInvalidBase;
                         }
@@ -259,73 +314,91 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
             }
 
             // ---- dense arithmetic, one replica (= one pipeline unit) at a time ----
-#pragma unroll
+            // (unrolled only for few replicas: beyond that the loop body no longer
+            // fits the instruction cache and fetch stalls cost more than the
+            // loop overhead saves)
+#pragma unroll(R <= 4 ? R : 1)
             for (int i = 0; i < R; ++i) {
                 cp_async_wait<NST - 2>();
-                issue_unit<R>(P, sd, pf, stage_base + ((n + NST - 1) % NST) * kUnitBytes, lane, n_warps);
+                issue_unit<R>(pf, P, sd, stage_base + ((n + NST - 1) % NST) * kUnitBytes, lane, n_warps);
                 const unsigned char *slot = my + (n % NST) * kUnitBytes + lane * 16;
                 ++n;
-                if (active) {
-                    const float4 w4 = *reinterpret_cast<const float4 *>(slot);
-                    const float4 g4 = *reinterpret_cast<const float4 *>(slot + 512);
-                    const float4 m4 = *reinterpret_cast<const float4 *>(slot + 1024);
-                    const float4 v4 = *reinterpret_cast<const float4 *>(slot + 1536);
-                    const uint64_t off = (uint64_t)i * stride + mu;
-                    const float w[4] = {w4.x, w4.y, w4.z, w4.w};
-                    const float g[4] = {g4.x, g4.y, g4.z, g4.w};
-                    float m[4] = {m4.x, m4.y, m4.z, m4.w};
-                    float v[4] = {v4.x, v4.y, v4.z, v4.w};
-                    float wh[4], wn[4];
+                float wn[V][4], wo[V][4];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        adamw(P, w[c], g[c], m[c], v[c], wh[c]);
-                        wn[c] = wh[c];
+                for (int h = 0; h < V; ++h) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) { wn[h][c] = 0.f; wo[h][c] = 0.f; }
+                    const uint64_t mu = mu0 + (uint64_t)h * 128;
+                    if (mu < N) {
+                        const float4 w4 = *reinterpret_cast<const float4 *>(slot + (0 * V + h) * 512);
+                        const float4 g4 = *reinterpret_cast<const float4 *>(slot + (1 * V + h) * 512);
+                        const float4 m4 = *reinterpret_cast<const float4 *>(slot + (2 * V + h) * 512);
+                        const float4 v4 = *reinterpret_cast<const float4 *>(slot + (3 * V + h) * 512);
+                        const uint64_t off = (uint64_t)i * stride + mu;
+                        const float g[4] = {g4.x, g4.y, g4.z, g4.w};
+                        float m[4] = {m4.x, m4.y, m4.z, m4.w};
+                        float v[4] = {v4.x, v4.y, v4.z, v4.w};
+                        wo[h][0] = w4.x; wo[h][1] = w4.y; wo[h][2] = w4.z; wo[h][3] = w4.w;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) adamw(P, wo[h][c], g[c], m[c], v[c], wn[h][c]);
+                        st_stream(st.M + off, m);
+                        st_stream(st.V + off, v);
                     }
-                    st_stream(st.M + off, m);
-                    st_stream(st.V + off, v);
+                }
 
-                    if (sm) {   // hand w^ and w^{t-1} of selected coordinates to the stash
+                if (sm) {   // hand w^ and w^{t-1} of selected coordinates to the stash
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if ((sm >> j) & 1u) {
-                                const uint32_t r = uexcl + __popc(um & ((1u << j) - 1u));
-                                st_what[r * R + i] = wh[j];
-                                st_wold[r * R + i] = w[j];
-                            }
+                    for (int j = 0; j < NB; ++j) {
+                        if ((sm >> j) & 1u) {
+                            const uint32_t r = uexcl + __popc(um & ((1u << j) - 1u));
+                            st_what[r * R + i] = wn[j >> 2][j & 3];
+                            st_wold[r * R + i] = wo[j >> 2][j & 3];
                         }
                     }
-                    if (om) {   // stash full: this lane does the sparse work itself
+                }
+                if (om) {   // stash full: this lane does the sparse work itself
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if ((om >> j) & 1u) {
-                                const uint32_t below = (1u << j) - 1u;
-                                if ((cm >> j) & 1u) {
-                                    const uint64_t ce = (uint64_t)(cfirst + __popc(cm & below)) * R;
-                                    float old[R];
-                                    load_replicas<R>(ring_cons + ce, old);
-                                    float a = old[0];
+                    for (int j = 0; j < NB; ++j) {
+                        if ((om >> j) & 1u) {
+                            const uint32_t below = (1u << j) - 1u;
+                            const float whj = wn[j >> 2][j & 3];
+                            if ((cm >> j) & 1u) {
+                                const uint64_t ce = (uint64_t)(cfirst + __popc(cm & below)) * R;
+                                float old[R];
+                                load_replicas<R>(ring_cons + ce, old);
+                                float a = old[0];
 #pragma unroll
-                                    for (int q = 1; q < R; ++q) a = __fadd_rn(a, old[q]);
-                                    const float abar = __fdiv_rn(a, P.Rf);
-                                    float *dp = st.D + (mu + j) * R + i;
-                                    const float diff = __fsub_rn(wh[j], old[i]);
-                                    const float dn = __fadd_rn(__fmul_rn(P.oml, *dp), __fmul_rn(P.lam, diff));
-                                    *dp = dn;
-                                    wn[j] = __fadd_rn(abar, dn);
-                                }
-                                if ((pm >> j) & 1u)
-                                    ring_prod[(uint64_t)(pfirst + __popc(pm & below)) * R + i] = wh[j];
+                                for (int q = 1; q < R; ++q) a = __fadd_rn(a, old[q]);
+                                const float abar = __fdiv_rn(a, P.Rf);
+                                float *dp = st.D + (mu0 + (uint64_t)(j >> 2) * 128 + (j & 3)) * R + i;
+                                float old_i = old[0];
+#pragma unroll
+                                for (int q = 1; q < R; ++q) old_i = (q == i) ? old[q] : old_i;
+                                const float diff = __fsub_rn(whj, old_i);
+                                const float dn = __fadd_rn(__fmul_rn(P.oml, *dp), __fmul_rn(P.lam, diff));
+                                *dp = dn;
+                                wn[j >> 2][j & 3] = __fadd_rn(abar, dn);
                             }
+                            if ((pm >> j) & 1u)
+                                ring_prod[(uint64_t)(pfirst + __popc(pm & below)) * R + i] = whj;
                         }
                     }
+                }
 
-                    st_stream(st.W + off, wn);
-                    if (has_look) {   // Section 2.2: extrapolate the last update direction
-                        float lk[4];
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            lk[c] = __fadd_rn(wn[c], __fmul_rn(delta, __fsub_rn(wn[c], w[c])));
-                        st_stream(st.LOOK + off, lk);
+                for (int h = 0; h < V; ++h) {
+                    const uint64_t mu = mu0 + (uint64_t)h * 128;
+                    if (mu < N) {
+                        const uint64_t off = (uint64_t)i * stride + mu;
+                        st_stream(st.W + off, wn[h]);
+                        if (has_look) {   // Section 2.2: extrapolate the last update direction
+                            float lk[4];
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                lk[c] = __fadd_rn(wn[h][c],
+                                                  __fmul_rn(delta, __fsub_rn(wn[h][c], wo[h][c])));
+                            st_stream(st.LOOK + off, lk);
+                        }
                     }
                 }
             }
@@ -335,7 +408,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
             for (uint32_t r0 = 0; r0 < n_s; r0 += 32) {
                 const uint32_t q = r0 + lane;
                 if (q < n_s) {
-                    if (r0 != 0) {   // second round (stash of 64): loads were not issued ahead
+                    if (r0 != 0) {   // later rounds: loads were not issued ahead
                         e_coord = st_coord[q];
                         e_c = st_cidx[q];
                         e_p = st_pidx[q];
