@@ -187,6 +187,34 @@ int asyncmesh_subset_mask(asyncmesh *h, uint32_t stage, uint64_t step,
  */
 int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *out_host);
 
+/*
+ * The same quantity for callers that cannot let the library allocate (the paper
+ * has no counterpart: this is a packaging variant of the call above, not part
+ * of the method).  Meant for hosts whose GPU memory is entirely owned by their
+ * own pool, for loops that must not hit the device-wide synchronisation an
+ * allocation may cause, and for hooks that run where the process may not grow:
+ * it calls no cudaMalloc / cudaFree and no allocating library routine.  The
+ * reduction's scratch (per-block partial sums) is a fixed 33 KB array inside
+ * the library image, present on every GPU that loads the library until the
+ * process exits.
+ *   w_device    device, [R][row_stride] fp32 (e.g. from asyncmesh_lookahead_weights
+ *               with delay 0), read-only, caller-owned
+ *   n           coordinates per row, 1 .. 2^28 (65536 per block x 4096 blocks of
+ *               scratch); larger n is rejected with INVALID_ARG and a message:
+ *               split the rows and add the partial results
+ *   out_host    host, receives sum_i ||w_i - wbar||^2 over the n coordinates
+ *   device, stream   where to run; the call waits for the stream before returning
+ * The first call on a device also looks up the scratch array's device address;
+ * make that first call before any stream capture.  All calls share the one
+ * array and it keeps the last call's contents (every slot a call reads it has
+ * written first, so nothing needs clearing); two calls whose kernels overlap on
+ * the GPU (different streams, different threads) race on it and must be
+ * serialised by the caller.
+ */
+int asyncmesh_consensus_error_noalloc(int device, void *stream, const float *w_device,
+                                      uint32_t R, uint64_t n, uint64_t row_stride,
+                                      double *out_host);
+
 /* Steps taken so far. */
 int asyncmesh_step_count(const asyncmesh *h, uint64_t *t);
 

@@ -7,6 +7,7 @@ from .binding import (AsyncMesh, AsyncMeshError, TorchAllocator, asyncmesh_creat
                       asyncmesh_destroy, asyncmesh_init_params, asyncmesh_step,
                       asyncmesh_step_ex, asyncmesh_step_host, asyncmesh_lookahead_weights,
                       asyncmesh_read_params, asyncmesh_read_state, asyncmesh_subset_mask,
-                      asyncmesh_consensus_error, asyncmesh_debug_philox,
+                      asyncmesh_consensus_error, asyncmesh_consensus_error_noalloc,
+                      asyncmesh_debug_philox,
                       asyncmesh_last_error, load)
 from .layouts import DEFAULT_HP, llama_stage_numel, workloads  # noqa: F401

@@ -70,6 +70,8 @@ SIGNATURES = {
     "asyncmesh_read_state": (_int, [_vp, _u32, _int, _i32, _vp, _u64, _int]),
     "asyncmesh_subset_mask": (_int, [_vp, _u32, _u64, _vp]),
     "asyncmesh_consensus_error": (_int, [_vp, _u32, ctypes.POINTER(ctypes.c_double)]),
+    "asyncmesh_consensus_error_noalloc": (_int, [_int, _vp, _vp, _u32, _u64, _u64,
+                                                 ctypes.POINTER(ctypes.c_double)]),
     "asyncmesh_step_count": (_int, [_vp, ctypes.POINTER(_u64)]),
     "asyncmesh_min_bytes_last_step": (_int, [_vp, ctypes.POINTER(_u64)]),
     "asyncmesh_status": (_int, [_vp]),
@@ -352,6 +354,17 @@ def asyncmesh_subset_mask(h: AsyncMesh, stage, step):
 
 def asyncmesh_consensus_error(h: AsyncMesh, stage):
     return h.consensus_error(stage)
+
+
+def asyncmesh_consensus_error_noalloc(w_device: int, R: int, n: int, row_stride: int,
+                                      device: int = 0, stream: int = 0) -> float:
+    """Consensus error of the rows at device address ``w_device`` through the entry
+    point that allocates nothing (its scratch is a fixed array inside the library,
+    good for n <= 2**28).  For callers that must not trigger an allocation."""
+    out = ctypes.c_double()
+    _check(load().asyncmesh_consensus_error_noalloc(device, stream, w_device, R, n, row_stride,
+                                                    ctypes.byref(out)))
+    return float(out.value)
 
 
 def asyncmesh_debug_philox(ctr: np.ndarray, key: np.ndarray, device: int = 0) -> np.ndarray:

@@ -795,3 +795,105 @@ extern "C" int asyncmesh_debug_philox(int device, const uint32_t *ctr_host, cons
     return ASYNCMESH_OK;
 }
 
+
+// ---------------------------------------------------------------------------
+// consensus error without any allocation
+// ---------------------------------------------------------------------------
+//
+// Some callers cannot take an entry point that allocates: a host that has handed
+// all of the GPU's memory to its own pool (a raw cudaMalloc would fail or eat
+// into a reserve it does not own), a control loop that must not hit the
+// device-wide synchronisation an allocation can cause, a monitoring hook that
+// runs where the process is not allowed to grow.  For them the reduction's
+// scratch lives in the library image itself: a fixed array in device memory that
+// every GPU holds from the moment it loads the library until the process exits.
+
+constexpr uint32_t kNoAllocTile = 1u << 16;        // coordinates one block reduces
+constexpr uint32_t kNoAllocMaxBlocks = 4096;       // => at most 2^28 coordinates per call
+constexpr uint64_t kNoAllocMaxCoords = (uint64_t)kNoAllocTile * kNoAllocMaxBlocks;
+
+// per-block partial sums, then the total in the last slot (33 KB per GPU)
+static __device__ __align__(256) double g_noalloc_scratch[kNoAllocMaxBlocks + 1];
+
+// In host code `g_noalloc_scratch` is only a stand-in for the device array; the
+// address kernels may use is looked up once per device and kept here.
+static double *g_noalloc_ptr[64] = {nullptr};
+
+__global__ void consensus_partial_kernel(const float *W, uint32_t R, uint64_t stride, uint64_t N,
+                                         double *partial)
+{
+    const uint64_t begin = (uint64_t)blockIdx.x * kNoAllocTile;
+    const uint64_t end = begin + kNoAllocTile < N ? begin + kNoAllocTile : N;
+    double acc = 0.0;
+    for (uint64_t mu = begin + threadIdx.x; mu < end; mu += blockDim.x) {
+        double mean = 0.0;
+        for (uint32_t i = 0; i < R; ++i) mean += (double)W[(uint64_t)i * stride + mu];
+        mean /= (double)R;
+        for (uint32_t i = 0; i < R; ++i) {
+            const double e = (double)W[(uint64_t)i * stride + mu] - mean;
+            acc += e * e;
+        }
+    }
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+    __shared__ double part[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) part[warp] = acc;
+    __syncthreads();
+    if (warp == 0) {
+        acc = lane < (int)(blockDim.x >> 5) ? part[lane] : 0.0;
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+        if (lane == 0) partial[blockIdx.x] = acc;   // every slot in use is overwritten: no clearing needed
+    }
+}
+
+__global__ void consensus_final_kernel(const double *partial, uint32_t n, double *total)
+{
+    double acc = 0.0;
+    for (uint32_t k = threadIdx.x; k < n; k += blockDim.x) acc += partial[k];
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+    __shared__ double part[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) part[warp] = acc;
+    __syncthreads();
+    if (warp == 0) {
+        acc = lane < (int)(blockDim.x >> 5) ? part[lane] : 0.0;
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+        if (lane == 0) *total = acc;
+    }
+}
+
+extern "C" int asyncmesh_consensus_error_noalloc(int device, void *stream, const float *w_device,
+                                                 uint32_t R, uint64_t n, uint64_t row_stride,
+                                                 double *out_host)
+{
+    if (!w_device || !out_host)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "consensus_error_noalloc: NULL argument");
+    if (R < 1 || n < 1 || row_stride < n)
+        return fail(ASYNCMESH_ERR_INVALID_ARG,
+                    "consensus_error_noalloc: need R >= 1, n >= 1, row_stride >= n");
+    if (n > kNoAllocMaxCoords)
+        return fail(ASYNCMESH_ERR_INVALID_ARG,
+                    "consensus_error_noalloc: n = %llu exceeds the built-in scratch (at most %llu "
+                    "coordinates per call; split the rows and add the results)",
+                    (unsigned long long)n, (unsigned long long)kNoAllocMaxCoords);
+    if (device < 0 || device >= 64)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "consensus_error_noalloc: device %d outside 0..63", device);
+    DeviceScope scope(device);
+    if (!scope.ok) return fail(ASYNCMESH_ERR_CUDA, "consensus_error_noalloc: cudaSetDevice(%d) failed", device);
+    if (!g_noalloc_ptr[device]) {   // first call on this device: find the array's device address
+        double *ptr = nullptr;
+        CU_TRY(cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch));
+        g_noalloc_ptr[device] = ptr;
+    }
+    double *scratch = g_noalloc_ptr[device];
+    const uint32_t blocks = (uint32_t)((n + kNoAllocTile - 1) / kNoAllocTile);
+    cudaStream_t st = (cudaStream_t)stream;
+    consensus_partial_kernel<<<blocks, 256, 0, st>>>(w_device, R, row_stride, n, scratch);
+    CU_TRY(cudaGetLastError());
+    consensus_final_kernel<<<1, 256, 0, st>>>(scratch, blocks, scratch + kNoAllocMaxBlocks);
+    CU_TRY(cudaGetLastError());
+    CU_TRY(cudaMemcpyAsync(out_host, scratch + kNoAllocMaxBlocks, sizeof(double),
+                           cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    return ASYNCMESH_OK;
+}
