@@ -171,6 +171,10 @@ int asyncmesh_read_params(asyncmesh *h, uint32_t stage, int32_t replica,
 int asyncmesh_read_state(asyncmesh *h, uint32_t stage, int which, int32_t replica,
                          float *dst, uint64_t n, int dst_on_device);
 
+/* The same for coordinates first .. first+count-1 of the row only. */
+int asyncmesh_read_state_range(asyncmesh *h, uint32_t stage, int which, int32_t replica,
+                               uint64_t first, uint64_t count, float *dst, int dst_on_device);
+
 /*
  * Membership of the subset S_stage^step as the device computes it: bit (mu & 7)
  * of bitmap_host[mu >> 3] is coordinate mu; (numel + 7) / 8 bytes, host memory.

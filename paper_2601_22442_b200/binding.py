@@ -68,6 +68,7 @@ SIGNATURES = {
                                            ctypes.POINTER(_u64)]),
     "asyncmesh_read_params": (_int, [_vp, _u32, _i32, _vp, _u64, _int]),
     "asyncmesh_read_state": (_int, [_vp, _u32, _int, _i32, _vp, _u64, _int]),
+    "asyncmesh_read_state_range": (_int, [_vp, _u32, _int, _i32, _u64, _u64, _vp, _int]),
     "asyncmesh_subset_mask": (_int, [_vp, _u32, _u64, _vp]),
     "asyncmesh_consensus_error": (_int, [_vp, _u32, ctypes.POINTER(ctypes.c_double)]),
     "asyncmesh_consensus_error_noalloc": (_int, [_int, _vp, _vp, _u32, _u64, _u64,
@@ -278,6 +279,18 @@ class AsyncMesh:
                                            dst.ctypes.data, n, 0))
         return dst
 
+    def read_state_range(self, stage: int, which: str, replica: int, first: int,
+                         count: int) -> np.ndarray:
+        dst = np.empty(count, dtype=np.float32)
+        _check(load().asyncmesh_read_state_range(self._h, stage, STATE[which], replica, first,
+                                                 count, dst.ctypes.data, 0))
+        return dst
+
+    def get_range(self, stage: int, which: str, first: int, count: int) -> np.ndarray:
+        """All replicas of one state array on a coordinate range: [R, count]."""
+        return np.stack([self.read_state_range(stage, which, i, first, count)
+                         for i in range(self.R)])
+
     def get(self, stage: int, which: str) -> np.ndarray:
         """All replicas of one state array: [R, numel[stage]]."""
         return np.stack([self.read_state(stage, which, i) for i in range(self.R)])
@@ -346,6 +359,10 @@ def asyncmesh_read_params(h: AsyncMesh, stage, replica=-1, out=None):
 
 def asyncmesh_read_state(h: AsyncMesh, stage, which, replica):
     return h.read_state(stage, which, replica)
+
+
+def asyncmesh_read_state_range(h: AsyncMesh, stage, which, replica, first, count):
+    return h.read_state_range(stage, which, replica, first, count)
 
 
 def asyncmesh_subset_mask(h: AsyncMesh, stage, step):

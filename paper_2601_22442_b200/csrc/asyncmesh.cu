@@ -156,12 +156,13 @@ __global__ void subset_bitmap_kernel(SubsetRule rule, uint32_t stage, uint32_t s
     }
 }
 
-// dst[mu] = D[mu][i]   (D is coordinate-major)
-__global__ void gather_column_kernel(const float *D, uint32_t R, uint32_t i, uint64_t N, float *dst)
+// dst[k] = D[first + k][i]   (D is coordinate-major)
+__global__ void gather_column_kernel(const float *D, uint32_t R, uint32_t i, uint64_t first,
+                                     uint64_t count, float *dst)
 {
-    for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
-         mu += (uint64_t)gridDim.x * blockDim.x)
-        dst[mu] = D[mu * R + i];
+    for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < count;
+         k += (uint64_t)gridDim.x * blockDim.x)
+        dst[k] = D[(first + k) * R + i];
 }
 
 // Replica mean in replica order, one division by (float) R.
@@ -672,16 +673,19 @@ static int deliver(asyncmesh *h, float *dst, uint64_t n, int dst_on_device, Prod
     return ASYNCMESH_OK;
 }
 
-extern "C" int asyncmesh_read_state(asyncmesh *h, uint32_t stage, int which, int32_t replica,
-                                    float *dst, uint64_t n, int dst_on_device)
+extern "C" int asyncmesh_read_state_range(asyncmesh *h, uint32_t stage, int which, int32_t replica,
+                                          uint64_t first, uint64_t count, float *dst,
+                                          int dst_on_device)
 {
     if (!h || !dst) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: NULL argument");
     if (stage >= h->S) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: stage %u >= S", stage);
     if (replica < 0 || replica >= (int32_t)h->R)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: replica %d outside 0..R-1", replica);
-    if (n != h->numel[stage])
-        return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: n = %llu, stage holds %llu",
-                    (unsigned long long)n, (unsigned long long)h->numel[stage]);
+    if (count < 1 || first >= h->numel[stage] || count > h->numel[stage] - first)
+        return fail(ASYNCMESH_ERR_INVALID_ARG,
+                    "read_state: range [%llu, +%llu) outside the stage's %llu coordinates",
+                    (unsigned long long)first, (unsigned long long)count,
+                    (unsigned long long)h->numel[stage]);
     DeviceScope scope(h->device);
     int rc = check_status(h, "read_state");
     if (rc != ASYNCMESH_OK) return rc;
@@ -696,15 +700,27 @@ extern "C" int asyncmesh_read_state(asyncmesh *h, uint32_t stage, int which, int
     default: return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: unknown selector %d", which);
     }
     if (row) {
-        CU_TRY(cudaMemcpyAsync(dst, row + (uint64_t)replica * d.stride, n * sizeof(float),
+        CU_TRY(cudaMemcpyAsync(dst, row + (uint64_t)replica * d.stride + first, count * sizeof(float),
                                dst_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost,
                                h->stream));
         CU_TRY(cudaStreamSynchronize(h->stream));
         return ASYNCMESH_OK;
     }
-    return deliver(h, dst, n, dst_on_device, [&](float *out) {
-        gather_column_kernel<<<grid_for(n, 256), 256, 0, h->stream>>>(d.D, h->R, (uint32_t)replica, n, out);
+    return deliver(h, dst, count, dst_on_device, [&](float *out) {
+        gather_column_kernel<<<grid_for(count, 256), 256, 0, h->stream>>>(d.D, h->R, (uint32_t)replica,
+                                                                         first, count, out);
     });
+}
+
+extern "C" int asyncmesh_read_state(asyncmesh *h, uint32_t stage, int which, int32_t replica,
+                                    float *dst, uint64_t n, int dst_on_device)
+{
+    if (!h || !dst) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: NULL argument");
+    if (stage >= h->S) return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: stage %u >= S", stage);
+    if (n != h->numel[stage])
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: n = %llu, stage holds %llu",
+                    (unsigned long long)n, (unsigned long long)h->numel[stage]);
+    return asyncmesh_read_state_range(h, stage, which, replica, 0, n, dst, dst_on_device);
 }
 
 extern "C" int asyncmesh_read_params(asyncmesh *h, uint32_t stage, int32_t replica, float *dst,
