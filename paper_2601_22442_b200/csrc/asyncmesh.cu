@@ -97,6 +97,7 @@ struct asyncmesh {
     double *scratch = nullptr;        // one double for reductions
 
     int mode = kSync;
+    bool pipelined = false;
     KernelChoice kernel;
     uint32_t n_slots = 0;
     uint32_t total_chunks = 0;
@@ -276,7 +277,10 @@ static bool stash_fits(double p)
 {
     const double q = 1.0 - (1.0 - p) * (1.0 - p);
     const double mean = kPipeSubCoords * q, sd = std::sqrt(kPipeSubCoords * q * (1.0 - q));
-    return mean + 4.0 * sd <= (double)PipeCfg<4>::kStash;
+#ifndef AM_STASH_SIGMAS
+#define AM_STASH_SIGMAS 4.0
+#endif
+    return mean + AM_STASH_SIGMAS * sd <= (double)PipeCfg<4>::kStash;
 }
 
 // ---------------------------------------------------------------------------
@@ -382,6 +386,10 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
     else { h->mode = kCompact; h->n_slots = h->tau + 1; }
 
+    // the compact ring has two kernels; which one is fixed for the handle's life
+    h->pipelined = h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
+                   (stash_fits(cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL));
+
     auto bail = [&](int code, const char *what) {
         release_all(h);
         delete h;
@@ -417,6 +425,10 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
             d.slot_floats = round_up(cap[s] * R, 64);
             d.chunk_base = (uint32_t *)zalloc((size_t)h->n_slots * d.n_chunks * sizeof(uint32_t));
             if (!d.chunk_base) return bail(ASYNCMESH_ERR_OOM, "out of device memory (ring index)");
+            if (h->pipelined) {
+                d.bitmap = (uint32_t *)zalloc((size_t)h->n_slots * d.n_chunks * 32 * sizeof(uint32_t));
+                if (!d.bitmap) return bail(ASYNCMESH_ERR_OOM, "out of device memory (subset masks)");
+            }
         } else if (h->mode == kDense) {
             d.slot_floats = h->stride[s] * R;
         }
@@ -441,9 +453,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
 
     // persistent grid: every SM filled to the kernel's occupancy
-    const bool pipelined = h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
-                           (stash_fits(cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL));
-    h->kernel = pick_kernel(R, h->mode, pipelined, S);
+    h->kernel = pick_kernel(R, h->mode, h->pipelined, S);
     int sms = 0, per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
     cudaError_t ke = cudaSuccess;

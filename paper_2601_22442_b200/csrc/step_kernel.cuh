@@ -54,6 +54,7 @@ struct StageDesc {
     float *LOOK;            // [R][stride]; == W when delta == 0
     float *ring;            // [n_slots][slot_floats]
     uint32_t *chunk_base;   // [n_slots][n_chunks]           (compact only)
+    uint32_t *bitmap;       // [n_slots][n_chunks][32] subset masks, lane-major (pipelined kernel only)
     uint64_t N, stride, slot_floats;
     uint32_t n_chunks;      // ceil(N / 1024)
     uint32_t chunk_begin;   // first chunk of this stage in the global list

@@ -55,6 +55,10 @@ __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gptr)
                  : "memory");
 }
+__device__ __forceinline__ void st_keep(float *p, const float (&x)[4])
+{
+    __stcg(reinterpret_cast<float4 *>(p), make_float4(x[0], x[1], x[2], x[3]));
+}
 __device__ __forceinline__ void cp_async_commit()
 {
     asm volatile("cp.async.commit_group;\n" ::: "memory");
@@ -205,7 +209,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 #pragma unroll
     for (int q = 0; q < NST - 1; ++q)
         issue_unit<R>(pf, P, sd, stage_base + q * kUnitBytes, lane, n_warps);
-    uint32_t n = 0;   // units consumed so far
+    uint32_t rd = 0, wr = NST - 1;   // ring slot being consumed / being filled
 
     const bool consume = P.consume != 0u;
     uint32_t s = 0;
@@ -217,13 +221,19 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         const uint64_t c0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
         const int kmax = pipe_sub_iterations(N, chunk);
 
-        // position of this chunk in the consumed slot: ask early, use late
-        uint32_t cbase = 0;
-        if (consume) cbase = st.chunk_base[(uint64_t)P.cons_slot * st.n_chunks + chunk];
+        // position of this chunk in the consumed slot and the membership mask stored
+        // when that slot was produced: ask early, use late
+        uint32_t cbase = 0, cmask = 0;
+        const uint64_t word = (uint64_t)chunk * 32 + lane;
+        if (consume) {
+            cbase = st.chunk_base[(uint64_t)P.cons_slot * st.n_chunks + chunk];
+            cmask = st.bitmap[(uint64_t)P.cons_slot * st.n_chunks * 32 + word];
+        }
 
-        // ---- membership of this lane's 32 coordinates in S^t and S^{t-tau} ----
+        // ---- membership of this lane's 32 coordinates in S^t (S^{t-tau} was read
+        // above: the generator runs once per coordinate and step) ----
         // bit 4b + c  <->  coordinate c0 + 128 b + c; sub-iteration k owns bits NB*k ..
-        uint32_t pmask = 0, cmask = 0;
+        uint32_t pmask = 0;
 #pragma unroll 2
         for (int b = 0; b < 8; ++b) {   // 8 quads per lane and chunk
             const uint64_t mu = c0 + (uint64_t)b * 128;
@@ -232,8 +242,6 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                 const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
                 const uint32_t quad = (uint32_t)(mu >> 2);
                 pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * b);
-                if (consume)
-                    cmask |= (subset_bits(P.rule, st.stage_id, P.cons_step, quad) & valid) << (4 * b);
             }
         }
 
@@ -259,6 +267,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         }
         pbase = __shfl_sync(kFullMask, pbase, 0);
         if (pbase == kInvalidBase) pmask = 0;
+        st.bitmap[(uint64_t)P.prod_slot * st.n_chunks * 32 + word] = pmask;   // for step t + tau
         const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
         float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
         const float delta = st.delta;
@@ -320,9 +329,10 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 #pragma unroll(R <= 4 ? R : 1)
             for (int i = 0; i < R; ++i) {
                 cp_async_wait<NST - 2>();
-                issue_unit<R>(pf, P, sd, stage_base + ((n + NST - 1) % NST) * kUnitBytes, lane, n_warps);
-                const unsigned char *slot = my + (n % NST) * kUnitBytes + lane * 16;
-                ++n;
+                issue_unit<R>(pf, P, sd, stage_base + wr * kUnitBytes, lane, n_warps);
+                const unsigned char *slot = my + rd * kUnitBytes + lane * 16;
+                rd = (rd + 1 == NST) ? 0 : rd + 1;
+                wr = (wr + 1 == NST) ? 0 : wr + 1;
                 float wn[V][4], wo[V][4];
 #pragma unroll
                 for (int h = 0; h < V; ++h) {
@@ -390,14 +400,16 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     const uint64_t mu = mu0 + (uint64_t)h * 128;
                     if (mu < N) {
                         const uint64_t off = (uint64_t)i * stride + mu;
-                        st_stream(st.W + off, wn[h]);
+                        // w and the look-ahead stay in L2 with normal priority: the few
+                        // selected coordinates of these lines are patched a moment later
+                        st_keep(st.W + off, wn[h]);
                         if (has_look) {   // Section 2.2: extrapolate the last update direction
                             float lk[4];
 #pragma unroll
                             for (int c = 0; c < 4; ++c)
                                 lk[c] = __fadd_rn(wn[h][c],
                                                   __fmul_rn(delta, __fsub_rn(wn[h][c], wo[h][c])));
-                            st_stream(st.LOOK + off, lk);
+                            st_keep(st.LOOK + off, lk);
                         }
                     }
                 }
