@@ -51,7 +51,7 @@ def lib() -> ctypes.CDLL:
         dbl, vp = ctypes.c_double, ctypes.c_void_p
         L.am_oracle_create.restype = vp
         L.am_oracle_create.argtypes = [u32, u32, vp, vp, dbl, u32, dbl, dbl, dbl,
-                                       dbl, dbl, dbl, u64, vp]
+                                       dbl, dbl, dbl, u64, vp, u32]
         L.am_oracle_destroy.restype = None
         L.am_oracle_destroy.argtypes = [vp]
         L.am_oracle_init_params.restype = ctypes.c_int
@@ -112,7 +112,7 @@ class Oracle:
                  beta2: float = 0.95, eps: float = 1e-8,
                  weight_decay: float = 0.1, seed: int = 0x5EED,
                  lookahead_delay: Optional[Sequence[int]] = None,
-                 coord_base: Optional[Sequence[int]] = None):
+                 coord_base: Optional[Sequence[int]] = None, avg_interval: int = 1):
         self.R, self.S, self.tau = int(R), len(numel), int(tau)
         self.numel = [int(n) for n in numel]
         self.p, self.seed = float(p), int(seed)
@@ -124,7 +124,7 @@ class Oracle:
         self._h = lib().am_oracle_create(
             self.R, self.S, ne, cb, float(p), self.tau, float(ema_beta),
             float(lr), float(beta1), float(beta2), float(eps),
-            float(weight_decay), self.seed, dl)
+            float(weight_decay), self.seed, dl, int(avg_interval))
         if not self._h:
             raise ValueError("oracle: invalid configuration or out of memory")
 

@@ -26,6 +26,10 @@
  *           w_i^t = wbar + d_i
  *       and w_i^t = w^_i^t for mu outside S^{t-tau}; d is untouched there.
  *       Nothing is consumed while t <= tau (no average has arrived yet).
+ *       With an averaging interval K > 1 (end of Section 3.2: averaging "every K
+ *       steps") O3 runs only at steps t = K, 2K, ...; the steps in between are
+ *       purely local (w^t = w^).  tau is then a multiple of K, so the average
+ *       consumed at a round was launched at an earlier round.
  *   O4  pipeline look-ahead (Section 2.2): the last update direction
  *       (w^t - w^{t-1}) extrapolated by the stage's delay delta_j:
  *           look_i = w_i^t + delta_j (w_i^t - w_i^{t-1}).
@@ -57,6 +61,7 @@
 
 typedef struct am_oracle {
     uint32_t R, S, tau;
+    uint32_t K;           /* averaging interval: subsets are exchanged at steps t = K, 2K, ... */
     uint64_t *numel;      /* [S] coordinates held for stage j               */
     uint64_t *coord_base; /* [S] global index of local coordinate 0         */
     uint32_t *delay;      /* [S] look-ahead delay delta_j                   */
@@ -147,12 +152,14 @@ am_oracle *am_oracle_create(uint32_t R, uint32_t S, const uint64_t *numel,
                             const uint64_t *coord_base, double p, uint32_t tau,
                             double lambda, double lr, double beta1,
                             double beta2, double eps, double wd, uint64_t seed,
-                            const uint32_t *delay)
+                            const uint32_t *delay, uint32_t avg_interval)
 {
     if (R < 1 || S < 1 || !numel || p < 0.0 || p > 1.0) return NULL;
+    if (avg_interval < 1) avg_interval = 1;
+    if (tau % avg_interval != 0) return NULL;
     am_oracle *o = (am_oracle *)calloc(1, sizeof(am_oracle));
     if (!o) return NULL;
-    o->R = R; o->S = S; o->tau = tau;
+    o->R = R; o->S = S; o->tau = tau; o->K = avg_interval;
     o->p = p; o->lambda = lambda; o->lr = lr; o->beta1 = beta1;
     o->beta2 = beta2; o->eps = eps; o->wd = wd; o->seed = seed;
     o->thresh = am_oracle_threshold(p);
@@ -248,7 +255,7 @@ int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
         }
 
         /* O3: delayed sparse averaging with EMA staleness correction */
-        const int consuming = t > tau;
+        const int consuming = (t % o->K == 0) && t > tau;   /* an averaging round with an arrival */
         const uint64_t u_step = t - tau;   /* only meaningful if consuming */
         const float *Hold = o->H[s] + (u_step % (tau + 1)) * (uint64_t)R * N;
         for (uint64_t mu = 0; mu < N; ++mu) {

@@ -31,7 +31,7 @@ def in_subset(seed, p, stage, step, mu):
 
 
 def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
-        stage=0):
+        stage=0, interval=1):
     """grads[t-1][i][mu] for t = 1..T.  Returns a list of per-step records."""
     T = len(grads)
     w = [[ft(w0[mu]) for mu in range(N)] for _ in range(R)]
@@ -62,7 +62,9 @@ def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
         hist[t] = what
         subsets[t] = {mu for mu in range(N) if in_subset(seed, p, stage, t, mu)}
         for mu in range(N):
-            if t - tau >= 1 and mu in subsets[t - tau]:
+            # averaging rounds are the steps K, 2K, ...; an average launched at round
+            # t - tau is consumed at round t
+            if t % interval == 0 and t - tau >= 1 and mu in subsets[t - tau]:
                 old = hist[t - tau]
                 acc = old[0][mu]
                 for i in range(1, R):

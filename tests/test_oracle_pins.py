@@ -350,6 +350,32 @@ def test_bruteforce_trace_second_stage_uses_its_own_subset():
     assert (o.get(0, "w") != o.get(1, "w")).any()
 
 
+@pytest.mark.parametrize("K,tau", [(2, 2), (3, 0), (2, 4), (4, 4)])
+def test_bruteforce_trace_with_averaging_interval(K, tau):
+    # averaging every K steps: the steps in between are purely local
+    R, N, T, seed = 3, 16, 13, 0x77
+    w0, grads = rand_setup(R, N, T, seed=21)
+    o = oracle.Oracle(R, [N], p=0.5, tau=tau, ema_beta=0.7, seed=seed,
+                      lookahead_delay=[2], avg_interval=K, **HP)
+    o.init_params(0, w0)
+    args = (R, N, 0.5, tau, 0.7, HP["lr"], HP["beta1"], HP["beta2"], HP["eps"],
+            HP["weight_decay"], seed, 2, w0, grads)
+    tr = bruteforce.run(np.float32, *args, interval=K)
+    changed = 0
+    for t in range(1, T + 1):
+        o.step([grads[t - 1]])
+        for name in ("w", "m", "v", "d", "look"):
+            assert (o.get(0, name).astype(np.float64) == tr[t - 1][name]).all(), (t, name)
+        same = (o.get(0, "w") == o.get(0, "what")).all()
+        if t % K != 0 or t <= tau:
+            assert same                      # a local step: nothing is averaged
+        else:
+            changed += int(not same)
+    assert changed > 0
+    with pytest.raises(ValueError):
+        oracle.Oracle(R, [N], p=0.5, tau=3, ema_beta=0.7, avg_interval=2)
+
+
 # ---- P9: elementwise independence ---------------------------------------------------
 
 def test_coordinate_slice_evolves_like_the_full_vector():
