@@ -87,7 +87,8 @@ typedef struct asyncmesh_config {
     uint64_t seed;                   /* Philox key of the subset rule                  */
     const uint32_t *lookahead_delay; /* host [S] or NULL (NULL: delta_j = S - 1 - j)   */
     int32_t device;                  /* CUDA device ordinal                            */
-    int32_t reserved;                /* must be 0                                      */
+    int32_t avg_interval;            /* K: subsets are exchanged every K-th step (end of
+                                        Section 3.2); 0 or 1 = every step; must divide tau */
     void *stream;                    /* cudaStream_t all work is issued on (NULL: the
                                         legacy default stream)                         */
     asyncmesh_alloc_fn alloc;        /* both NULL: cudaMalloc / cudaFree               */

@@ -39,7 +39,7 @@ class Config(ctypes.Structure):
         ("eps", ctypes.c_double), ("weight_decay", ctypes.c_double),
         ("seed", ctypes.c_uint64),
         ("lookahead_delay", ctypes.POINTER(ctypes.c_uint32)),
-        ("device", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("device", ctypes.c_int32), ("avg_interval", ctypes.c_int32),
         ("stream", ctypes.c_void_p),
         ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_ctx", ctypes.c_void_p),
     ]
@@ -149,7 +149,7 @@ class AsyncMesh:
                  seed: int = 0x5EED, lookahead_delay: Optional[Sequence[int]] = None,
                  device: int = 0, stream: Optional[int] = None,
                  allocator: Optional[TorchAllocator] = None,
-                 use_torch_allocator: bool = True, flags: int = 0):
+                 use_torch_allocator: bool = True, flags: int = 0, avg_interval: int = 1):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("asyncmesh needs a CUDA device; there is no CPU path")
@@ -175,7 +175,7 @@ class AsyncMesh:
         cfg.eps, cfg.weight_decay, cfg.seed = float(eps), float(weight_decay), int(seed)
         if dl is not None:
             cfg.lookahead_delay = ctypes.cast(dl, ctypes.POINTER(ctypes.c_uint32))
-        cfg.device, cfg.reserved, cfg.stream = self.device, 0, stream
+        cfg.device, cfg.avg_interval, cfg.stream = self.device, int(avg_interval), stream
         if self.allocator is not None:
             cfg.alloc, cfg.free = self.allocator.alloc_cb, self.allocator.free_cb
         h = _vp()

@@ -77,6 +77,8 @@ struct KernelChoice {
 
 struct asyncmesh {
     uint32_t R = 0, S = 0, tau = 0;
+    uint32_t K = 1;                   // averaging interval in steps; tau is a multiple of it
+    uint32_t lag = 0;                 // tau / K: averaging rounds between launch and arrival
     double p = 0, ema_beta = 0, lr = 0, beta1 = 0, beta2 = 0, eps = 0, wd = 0;
     uint64_t seed = 0;
     int device = 0;
@@ -312,8 +314,13 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if (!(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: betas must lie in [0, 1)");
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
-                        ASYNCMESH_FLAG_PIPELINED_KERNEL)) != 0 || cfg->reserved != 0)
-        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags, or reserved is not 0");
+                        ASYNCMESH_FLAG_PIPELINED_KERNEL)) != 0)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
+    const uint32_t K = cfg->avg_interval < 1 ? 1u : (uint32_t)cfg->avg_interval;
+    if (cfg->avg_interval < 0 || cfg->tau % K != 0)
+        return fail(ASYNCMESH_ERR_INVALID_ARG,
+                    "create: avg_interval = %d must be >= 0 and divide tau = %u", cfg->avg_interval,
+                    cfg->tau);
     if ((cfg->alloc == nullptr) != (cfg->free == nullptr))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: give both alloc and free, or neither");
     for (uint32_t s = 0; s < cfg->S; ++s)
@@ -334,6 +341,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     asyncmesh *h = new (std::nothrow) asyncmesh();
     if (!h) return fail(ASYNCMESH_ERR_OOM, "create: host allocation failed");
     h->R = cfg->R; h->S = cfg->S; h->tau = cfg->tau;
+    h->K = K; h->lag = cfg->tau / K;
     h->p = cfg->p; h->ema_beta = cfg->ema_beta; h->lr = cfg->lr;
     h->beta1 = cfg->beta1; h->beta2 = cfg->beta2; h->eps = cfg->eps; h->wd = cfg->weight_decay;
     h->seed = cfg->seed; h->device = cfg->device; h->stream = (cudaStream_t)cfg->stream;
@@ -368,8 +376,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         if (c > (double)N) c = (double)N;
         cap[s] = (uint64_t)c;
         if ((cfg->flags & ASYNCMESH_FLAG_SMALL_RING) && h->tau > 0) cap[s] = cap[s] / 8 + 1;
-        compact_total += (long double)(h->tau + 1) * cap[s];
-        dense_total += (long double)h->tau * h->stride[s];
+        compact_total += (long double)(h->lag + 1) * cap[s];
+        dense_total += (long double)h->lag * h->stride[s];
         h->sd[s].n_chunks = (uint32_t)((N + kWarpChunk - 1) / kWarpChunk);
         h->sd[s].chunk_begin = (uint32_t)chunks;
         chunks += h->sd[s].n_chunks;
@@ -382,9 +390,9 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if (h->tau == 0) { h->mode = kSync; h->n_slots = 0; }
     else if (dense_total <= compact_total &&
              !(cfg->flags & (ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_PIPELINED_KERNEL))) {
-        h->mode = kDense; h->n_slots = h->tau;
+        h->mode = kDense; h->n_slots = h->lag;
     }
-    else { h->mode = kCompact; h->n_slots = h->tau + 1; }
+    else { h->mode = kCompact; h->n_slots = h->lag + 1; }
 
     // the compact ring has two kernels; which one is fixed for the handle's life
     h->pipelined = h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
@@ -551,13 +559,17 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.S = h->S;
     P.total_chunks = h->total_chunks;
     P.step = (uint32_t)t;
+    // averaging rounds are the steps K, 2K, ...; in between the step is purely local
+    const bool round = (t % h->K) == 0;
+    const uint64_t r = t / h->K;   // index of this round
     P.cons_step = (uint32_t)(t - h->tau);
-    P.consume = (h->mode != kSync && t > h->tau) ? 1u : 0u;
+    P.produce = round ? 1u : 0u;
+    P.consume = (h->mode != kSync && round && t > h->tau) ? 1u : 0u;
     if (h->mode == kCompact) {
-        P.prod_slot = (uint32_t)(t % (h->tau + 1));
-        P.cons_slot = (uint32_t)((t - h->tau) % (h->tau + 1));   // unused while t <= tau
+        P.prod_slot = (uint32_t)(r % (h->lag + 1));
+        P.cons_slot = (uint32_t)((r - h->lag) % (h->lag + 1));   // unused while t <= tau
     } else if (h->mode == kDense) {
-        P.prod_slot = P.cons_slot = (uint32_t)(t % h->tau);
+        P.prod_slot = P.cons_slot = (uint32_t)(r % h->lag);
     }
     P.rule = h->rule;
     // per-step scalars: double arithmetic, one rounding to fp32 each
@@ -574,7 +586,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.oml = (float)(1.0 - lam);
     P.Rf = (float)h->R;
 
-    if (h->mode == kCompact)   // the producing slot's cursors start this step at zero
+    if (h->mode == kCompact && round)   // the producing slot's cursors start this step at zero
         CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
                                h->S * sizeof(unsigned int), h->stream));
 
@@ -586,7 +598,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     double bytes = 0.0;
     for (uint32_t s = 0; s < h->S; ++s) {
         double per = 28.0 + (h->delay[s] ? 4.0 : 0.0);
-        if (h->mode != kSync) per += 4.0 * h->p + (P.consume ? 12.0 * h->p : 0.0);
+        if (h->mode != kSync && round) per += 4.0 * h->p + (P.consume ? 12.0 * h->p : 0.0);
         bytes += per * (double)h->R * (double)h->numel[s];
     }
     h->last_bytes = (uint64_t)bytes;

@@ -71,7 +71,8 @@ struct StepParams {
     const float *G[kMaxStages];  // gradients, [R][stride] each
     uint32_t S, total_chunks;
     uint32_t step, cons_step;    // t and t - tau
-    uint32_t consume;            // t > tau
+    uint32_t produce;            // this step is an averaging round: S^t is snapshotted
+    uint32_t consume;            // ... and the average launched at t - tau has arrived
     uint32_t prod_slot, cons_slot;
     SubsetRule rule;
     float b1, b2, omb1, omb2, ib1, ib2, eps, lr, lrwd, lam, oml, Rf;
@@ -158,7 +159,8 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
             const uint64_t left = N - mu;
             const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
             const uint32_t quad = (uint32_t)(mu >> 2);
-            pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * k);
+            if (P.produce)
+                pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * k);
             if (consume)
                 cmask |= (subset_bits(P.rule, st.stage_id, P.cons_step, quad) & valid) << (4 * k);
         }
@@ -178,7 +180,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                     atomicExch(P.status, kStatusRingOverflow);
                 }
             }
-            st.chunk_base[(uint64_t)P.prod_slot * st.n_chunks + chunk] = b;
+            if (P.produce) st.chunk_base[(uint64_t)P.prod_slot * st.n_chunks + chunk] = b;
             pbase = b;
         }
         pbase = __shfl_sync(kFullMask, pbase, 0);

@@ -241,7 +241,8 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                 const uint64_t left = N - mu;
                 const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
                 const uint32_t quad = (uint32_t)(mu >> 2);
-                pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * b);
+                if (P.produce)
+                    pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * b);
             }
         }
 
@@ -257,7 +258,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     atomicExch(P.status, kStatusRingOverflow);
                 }
             }
-            st.chunk_base[(uint64_t)P.prod_slot * st.n_chunks + chunk] = b;
+            if (P.produce) st.chunk_base[(uint64_t)P.prod_slot * st.n_chunks + chunk] = b;
             pbase = b;
         }
         if (consume) {
@@ -267,7 +268,8 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         }
         pbase = __shfl_sync(kFullMask, pbase, 0);
         if (pbase == kInvalidBase) pmask = 0;
-        st.bitmap[(uint64_t)P.prod_slot * st.n_chunks * 32 + word] = pmask;   // for step t + tau
+        if (P.produce)   // kept for step t + tau
+            st.bitmap[(uint64_t)P.prod_slot * st.n_chunks * 32 + word] = pmask;
         const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
         float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
         const float delta = st.delta;

@@ -41,7 +41,7 @@ def test_config_struct_matches_header_layout():
     assert offs["p"] == 16 and offs["tau"] == 24 and offs["flags"] == 28
     assert offs["ema_beta"] == 32 and offs["lr"] == 40 and offs["weight_decay"] == 72
     assert offs["seed"] == 80 and offs["lookahead_delay"] == 88
-    assert offs["device"] == 96 and offs["reserved"] == 100 and offs["stream"] == 104
+    assert offs["device"] == 96 and offs["avg_interval"] == 100 and offs["stream"] == 104
     assert offs["alloc"] == 112 and offs["free"] == 120 and offs["alloc_ctx"] == 128
     assert ctypes.sizeof(binding.Config) == 136
 
@@ -63,7 +63,8 @@ def _cfg(**over):
     (dict(R=0), "R ="), (dict(R=17), "R ="), (dict(S=0), "S ="), (dict(S=65), "S ="),
     (dict(p=-0.1), "p ="), (dict(p=1.5), "p ="), (dict(p=float("nan")), "p ="),
     (dict(tau=65), "tau"), (dict(ema_beta=1.01), "ema_beta"), (dict(lr=0.0), "lr"),
-    (dict(eps=0.0), "eps"), (dict(beta1=1.0), "betas"), (dict(flags=8), "flags"),
+    (dict(eps=0.0), "eps"), (dict(beta1=1.0), "betas"), (dict(tau=3, avg_interval=2), "avg_interval"),
+    (dict(avg_interval=-1), "avg_interval"), (dict(flags=8), "flags"),
 ])
 def test_create_rejects_bad_arguments_without_touching_a_device(lib, over, word):
     h = ctypes.c_void_p()

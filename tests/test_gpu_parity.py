@@ -26,11 +26,11 @@ def am():
 
 
 def make_pair(R, numel, p, tau, lam, delays=None, seed=0x5EED, hp=HP, same_init=True,
-              init_seed=0x1217, flags=0):
+              init_seed=0x1217, flags=0, avg_interval=1):
     o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
-                      lookahead_delay=delays, **hp)
+                      lookahead_delay=delays, avg_interval=avg_interval, **hp)
     g = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
-                       lookahead_delay=delays, flags=flags, **hp)
+                       lookahead_delay=delays, flags=flags, avg_interval=avg_interval, **hp)
     for s, n in enumerate(numel):
         if same_init:
             w0 = si.init_weights_host(init_seed, s, 0, n)
@@ -161,6 +161,15 @@ def test_ragged_stage_sizes():
     run_case(3, sizes, 0.2, 2, 0.7, steps=6, delays=[k % 3 for k in range(len(sizes))])
     run_case(2, sizes, 1.0, 2, 0.7, steps=6)
     run_case(4, sizes, 0.4, 0, 0.7, steps=3)
+
+
+@pytest.mark.parametrize("K,tau,p", [(2, 2, 0.05), (3, 6, 0.3), (2, 0, 0.3), (4, 4, 1.0), (2, 4, 0.7)])
+def test_averaging_interval(K, tau, p):
+    # subsets exchanged every K-th step only (all ring modes); in between purely local
+    from paper_2601_22442_b200 import binding
+    run_case(4, [5000, 1024 * 2 + 3], p, tau, 0.9, steps=4 * K + tau + 1, avg_interval=K)
+    run_case(3, [5000], p, tau, 0.9, steps=3 * K + tau + 1, avg_interval=K,
+             flags=binding.FLAG_DIRECT_KERNEL)
 
 
 @pytest.mark.parametrize("lam", [0.0, 1.0])
