@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.am_oracle_create.restype = vp
         L.am_oracle_create.argtypes = [u32, u32, vp, vp, dbl, u32, dbl, dbl, dbl,
                                        dbl, dbl, dbl, u64, vp, u32]
+        L.am_oracle_set_optimizer.restype = None
+        L.am_oracle_set_optimizer.argtypes = [vp, u32, dbl]
         L.am_oracle_destroy.restype = None
         L.am_oracle_destroy.argtypes = [vp]
         L.am_oracle_init_params.restype = ctypes.c_int
@@ -112,7 +114,8 @@ class Oracle:
                  beta2: float = 0.95, eps: float = 1e-8,
                  weight_decay: float = 0.1, seed: int = 0x5EED,
                  lookahead_delay: Optional[Sequence[int]] = None,
-                 coord_base: Optional[Sequence[int]] = None, avg_interval: int = 1):
+                 coord_base: Optional[Sequence[int]] = None, avg_interval: int = 1,
+                 optimizer: str = "adamw", momentum_decay: float = 4e-3):
         self.R, self.S, self.tau = int(R), len(numel), int(tau)
         self.numel = [int(n) for n in numel]
         self.p, self.seed = float(p), int(seed)
@@ -127,6 +130,8 @@ class Oracle:
             float(weight_decay), self.seed, dl, int(avg_interval))
         if not self._h:
             raise ValueError("oracle: invalid configuration or out of memory")
+        lib().am_oracle_set_optimizer(self._h, {"adamw": 0, "nadamw": 1}[optimizer],
+                                      float(momentum_decay))
 
     def close(self) -> None:
         if getattr(self, "_h", None):

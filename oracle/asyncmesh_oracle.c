@@ -14,6 +14,14 @@
  *       (first line of Eq. "sparta", Section 2.3).  The optimizer is the
  *       textbook decoupled-weight-decay Adam (AdamW) with bias correction;
  *       its moments m, v are local to a replica and never averaged.
+ *       Alternatively NAdamW, the optimizer the paper itself uses for
+ *       asynchronous pipelines (Appendix B.1: NAdamW, momentum 0.99): Adam with
+ *       Nesterov momentum (Dozat, 2016) and decoupled weight decay.  With
+ *       mu_t = beta1 (1 - 0.5 * 0.96^(t psi)) and PI_t = mu_1 ... mu_t:
+ *           w^ = w - lr wd w - lr (1 - mu_t)/(1 - PI_t)        g / (sqrt(v^) + eps)
+ *                            - lr mu_{t+1}/(1 - PI_t mu_{t+1}) m / (sqrt(v^) + eps)
+ *       (m, v updated first; v^ bias-corrected, m is not: the momentum schedule
+ *       takes that role).
  *   O2  snapshot of w^_i^t for the averaging launched at step t
  *       (Section 3.1: the average of step t arrives tau steps later; the
  *       appendix says the asynchronous setup is simulated by buffering).
@@ -62,6 +70,8 @@
 typedef struct am_oracle {
     uint32_t R, S, tau;
     uint32_t K;           /* averaging interval: subsets are exchanged at steps t = K, 2K, ... */
+    uint32_t optimizer;   /* 0 AdamW, 1 NAdamW                                                  */
+    double momentum_decay, mu_product; /* NAdam's momentum schedule and its running product      */
     uint64_t *numel;      /* [S] coordinates held for stage j               */
     uint64_t *coord_base; /* [S] global index of local coordinate 0         */
     uint32_t *delay;      /* [S] look-ahead delay delta_j                   */
@@ -206,6 +216,14 @@ int am_oracle_init_params(am_oracle *o, uint32_t stage, int32_t replica,
  * lambda_t / lr_t < 0 mean "use the constant given at creation"; otherwise
  * they replace it for this step (the paper decays both over training).
  */
+void am_oracle_set_optimizer(am_oracle *o, uint32_t optimizer, double momentum_decay)
+{
+    if (!o) return;
+    o->optimizer = optimizer;
+    o->momentum_decay = momentum_decay;
+    o->mu_product = 1.0;
+}
+
 int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
                       double lr_t)
 {
@@ -224,6 +242,13 @@ int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
     const float eps = (float)o->eps;
     const float lam = (float)lam_d, oml = (float)(1.0 - lam_d);
     const float Rf = (float)R;
+    /* NAdam's momentum schedule (scalars only; unused by AdamW) */
+    const double mu_t = o->beta1 * (1.0 - 0.5 * pow(0.96, (double)t * o->momentum_decay));
+    const double mu_n = o->beta1 * (1.0 - 0.5 * pow(0.96, (double)(t + 1) * o->momentum_decay));
+    if (o->mu_product == 0.0) o->mu_product = 1.0;
+    o->mu_product *= mu_t;
+    const float cg = (float)(lr_d * (1.0 - mu_t) / (1.0 - o->mu_product));
+    const float cm = (float)(lr_d * mu_n / (1.0 - o->mu_product * mu_n));
 
     for (uint32_t s = 0; s < o->S; ++s) {
         const uint64_t N = o->numel[s];
@@ -244,10 +269,17 @@ int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
                 const float mh = mk * ib1;
                 const float vh = vk * ib2;
                 const float den = sqrtf(vh) + eps;
-                const float u = mh / den;
                 const float wk = w[k];
                 float wh = wk - (lrwd * wk);   /* decoupled weight decay */
-                wh = wh - (lr * u);            /* Adam step              */
+                if (o->optimizer == 0) {
+                    const float u = mh / den;
+                    wh = wh - (lr * u);        /* Adam step              */
+                } else {
+                    const float ug = gk / den; /* Nesterov: gradient part ... */
+                    const float um = mk / den; /* ... and momentum part       */
+                    wh = wh - (cg * ug);
+                    wh = wh - (cm * um);
+                }
                 wprev[k] = wk;
                 what[k] = wh;
                 Hnow[k] = wh;

@@ -143,6 +143,37 @@ def test_adamw_constant_gradient_closed_form():
     assert np.abs(o.row(0, "w", 0) - expect).max() < 5e-6 * HP["lr"] * T
 
 
+def test_nadamw_against_torch_library():
+    # the paper's optimizer for asynchronous pipelines: NAdam with decoupled decay,
+    # momentum 0.99
+    R, N, T = 2, 1 << 13, 60
+    w0, grads = rand_setup(R, N, T)
+    hp = dict(HP, beta1=0.99)
+    o = oracle.Oracle(R, [N], p=0.0, tau=0, ema_beta=0.9, lookahead_delay=[0],
+                      optimizer="nadamw", **hp)
+    o.init_params(0, w0)
+    for g in grads:
+        o.step([g])
+    for i in range(R):
+        q = torch.nn.Parameter(torch.tensor(w0, dtype=torch.float64))
+        opt = torch.optim.NAdam([q], lr=hp["lr"], betas=(hp["beta1"], hp["beta2"]), eps=hp["eps"],
+                                weight_decay=hp["weight_decay"], momentum_decay=4e-3,
+                                decoupled_weight_decay=True)
+        for g in grads:
+            q.grad = torch.tensor(g[i], dtype=torch.float64)
+            opt.step()
+        st = opt.state[q]
+        assert np.abs(o.row(0, "w", i) - q.detach().numpy()).max() < 2e-7
+        assert np.abs(o.row(0, "m", i) - st["exp_avg"].numpy()).max() < 1e-9
+        assert relerr(o.row(0, "v", i), st["exp_avg_sq"].numpy()) < 2e-6
+    # and it is not AdamW
+    a = oracle.Oracle(R, [N], p=0.0, tau=0, ema_beta=0.9, lookahead_delay=[0], **hp)
+    a.init_params(0, w0)
+    for g in grads:
+        a.step([g])
+    assert np.abs(a.row(0, "w", 0) - o.row(0, "w", 0)).max() > 1e-5
+
+
 # ---- P2: p = 1, tau = 0 is "average everything every step" --------------------
 
 def test_full_sync_averaging_against_torch():
