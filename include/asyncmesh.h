@@ -45,6 +45,10 @@ extern "C" {
 #define ASYNCMESH_MAX_STAGES 64u
 #define ASYNCMESH_MAX_TAU 64u
 
+/* asyncmesh_config.optimizer */
+#define ASYNCMESH_OPT_ADAMW 0u
+#define ASYNCMESH_OPT_NADAMW 1u
+
 /* asyncmesh_config.flags */
 #define ASYNCMESH_FLAG_SMALL_RING 1u /* diagnostic: give each compact ring slot 1/8 of
                                         its normal capacity, so that the overflow
@@ -94,6 +98,13 @@ typedef struct asyncmesh_config {
     asyncmesh_alloc_fn alloc;        /* both NULL: cudaMalloc / cudaFree               */
     asyncmesh_free_fn free;
     void *alloc_ctx;
+    uint32_t optimizer;              /* ASYNCMESH_OPT_ADAMW (0) or ASYNCMESH_OPT_NADAMW: Adam with
+                                        Nesterov momentum and decoupled decay, the optimizer the
+                                        paper runs asynchronous pipelines with (Appendix B.1,
+                                        momentum beta1 = 0.99)                             */
+    uint32_t pad0;                   /* must be 0                                       */
+    double momentum_decay;           /* NAdamW: psi of mu_t = beta1 (1 - 0.5 * 0.96^(t psi));
+                                        0 selects the customary 0.004                   */
 } asyncmesh_config;
 
 /*

@@ -12,3 +12,4 @@ from .binding import (AsyncMesh, AsyncMeshError, TorchAllocator, asyncmesh_creat
                       asyncmesh_debug_philox,
                       asyncmesh_last_error, load)
 from .layouts import DEFAULT_HP, llama_stage_numel, workloads  # noqa: F401
+from .schedules import ema_coefficient, learning_rate  # noqa: F401

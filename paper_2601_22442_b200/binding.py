@@ -42,6 +42,8 @@ class Config(ctypes.Structure):
         ("device", ctypes.c_int32), ("avg_interval", ctypes.c_int32),
         ("stream", ctypes.c_void_p),
         ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_ctx", ctypes.c_void_p),
+        ("optimizer", ctypes.c_uint32), ("pad0", ctypes.c_uint32),
+        ("momentum_decay", ctypes.c_double),
     ]
 
 
@@ -149,7 +151,8 @@ class AsyncMesh:
                  seed: int = 0x5EED, lookahead_delay: Optional[Sequence[int]] = None,
                  device: int = 0, stream: Optional[int] = None,
                  allocator: Optional[TorchAllocator] = None,
-                 use_torch_allocator: bool = True, flags: int = 0, avg_interval: int = 1):
+                 use_torch_allocator: bool = True, flags: int = 0, avg_interval: int = 1,
+                 optimizer: str = "adamw", momentum_decay: float = 4e-3):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("asyncmesh needs a CUDA device; there is no CPU path")
@@ -176,6 +179,8 @@ class AsyncMesh:
         if dl is not None:
             cfg.lookahead_delay = ctypes.cast(dl, ctypes.POINTER(ctypes.c_uint32))
         cfg.device, cfg.avg_interval, cfg.stream = self.device, int(avg_interval), stream
+        cfg.optimizer = {"adamw": 0, "nadamw": 1}[optimizer]
+        cfg.pad0, cfg.momentum_decay = 0, float(momentum_decay)
         if self.allocator is not None:
             cfg.alloc, cfg.free = self.allocator.alloc_cb, self.allocator.free_cb
         h = _vp()

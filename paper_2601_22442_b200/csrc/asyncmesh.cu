@@ -77,6 +77,8 @@ struct KernelChoice {
 
 struct asyncmesh {
     uint32_t R = 0, S = 0, tau = 0;
+    uint32_t optimizer = 0;           // ASYNCMESH_OPT_*
+    double momentum_decay = 4e-3, mu_product = 1.0;   // NAdamW's momentum schedule
     uint32_t K = 1;                   // averaging interval in steps; tau is a multiple of it
     uint32_t lag = 0;                 // tau / K: averaging rounds between launch and arrival
     double p = 0, ema_beta = 0, lr = 0, beta1 = 0, beta2 = 0, eps = 0, wd = 0;
@@ -316,6 +318,9 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
                         ASYNCMESH_FLAG_PIPELINED_KERNEL)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
+    if (cfg->optimizer > ASYNCMESH_OPT_NADAMW || cfg->pad0 != 0 || !(cfg->momentum_decay >= 0.0))
+        return fail(ASYNCMESH_ERR_INVALID_ARG,
+                    "create: optimizer must be 0 (AdamW) or 1 (NAdamW), pad0 0, momentum_decay >= 0");
     const uint32_t K = cfg->avg_interval < 1 ? 1u : (uint32_t)cfg->avg_interval;
     if (cfg->avg_interval < 0 || cfg->tau % K != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG,
@@ -342,6 +347,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if (!h) return fail(ASYNCMESH_ERR_OOM, "create: host allocation failed");
     h->R = cfg->R; h->S = cfg->S; h->tau = cfg->tau;
     h->K = K; h->lag = cfg->tau / K;
+    h->optimizer = cfg->optimizer;
+    h->momentum_decay = cfg->momentum_decay > 0.0 ? cfg->momentum_decay : 4e-3;
     h->p = cfg->p; h->ema_beta = cfg->ema_beta; h->lr = cfg->lr;
     h->beta1 = cfg->beta1; h->beta2 = cfg->beta2; h->eps = cfg->eps; h->wd = cfg->weight_decay;
     h->seed = cfg->seed; h->device = cfg->device; h->stream = (cudaStream_t)cfg->stream;
@@ -585,6 +592,15 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.lam = (float)lam;
     P.oml = (float)(1.0 - lam);
     P.Rf = (float)h->R;
+    P.nesterov = h->optimizer == ASYNCMESH_OPT_NADAMW ? 1u : 0u;
+    double mu_product = h->mu_product;
+    if (P.nesterov) {   // mu_t, mu_{t+1} and the running product of the momentum schedule
+        const double mu_t = h->beta1 * (1.0 - 0.5 * std::pow(0.96, (double)t * h->momentum_decay));
+        const double mu_n = h->beta1 * (1.0 - 0.5 * std::pow(0.96, (double)(t + 1) * h->momentum_decay));
+        mu_product *= mu_t;
+        P.cg = (float)(lr * (1.0 - mu_t) / (1.0 - mu_product));
+        P.cm = (float)(lr * mu_n / (1.0 - mu_product * mu_n));
+    }
 
     if (h->mode == kCompact && round)   // the producing slot's cursors start this step at zero
         CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
@@ -593,6 +609,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     h->kernel.fn<<<h->grid, h->kernel.threads, h->kernel.smem, h->stream>>>(P);
     CU_TRY(cudaGetLastError());
     h->t = t;
+    h->mu_product = mu_product;
 
     // roofline numerator (see the header): bytes this step could not avoid
     double bytes = 0.0;

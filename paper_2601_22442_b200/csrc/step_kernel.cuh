@@ -76,6 +76,8 @@ struct StepParams {
     uint32_t prod_slot, cons_slot;
     SubsetRule rule;
     float b1, b2, omb1, omb2, ib1, ib2, eps, lr, lrwd, lam, oml, Rf;
+    uint32_t nesterov;           // 0: AdamW, 1: NAdamW
+    float cg, cm;                // NAdamW: weights of the gradient and momentum parts
 };
 
 __device__ __forceinline__ float4 ld_stream(const float *p)
@@ -87,8 +89,8 @@ __device__ __forceinline__ void st_stream(float *p, const float (&x)[4])
     __stcs(reinterpret_cast<float4 *>(p), make_float4(x[0], x[1], x[2], x[3]));
 }
 
-// AdamW with decoupled weight decay and bias correction, one rounding per
-// written operation (first line of Eq. "sparta": the local optimizer step).
+// The local optimizer step (first line of Eq. "sparta"), one rounding per written
+// operation: AdamW with decoupled weight decay and bias correction, or NAdamW.
 __device__ __forceinline__ void adamw(const StepParams &P, float w, float g, float &m,
                                       float &v, float &what)
 {
@@ -96,15 +98,18 @@ __device__ __forceinline__ void adamw(const StepParams &P, float w, float g, flo
     v = __fadd_rn(__fmul_rn(P.b2, v), __fmul_rn(P.omb2, __fmul_rn(g, g)));
     const float mh = __fmul_rn(m, P.ib1);
     const float vh = __fmul_rn(v, P.ib2);
-#ifdef AM_EXPERIMENT_FAST_MATH   // timing experiment only: not IEEE, breaks parity
-    const float den = __fadd_rn(__fmul_rn(vh, rsqrtf(vh)), P.eps);
-    const float u = __fdividef(mh, den);
-#else
     const float den = __fadd_rn(__fsqrt_rn(vh), P.eps);
-    const float u = __fdiv_rn(mh, den);
-#endif
     const float decayed = __fsub_rn(w, __fmul_rn(P.lrwd, w));
-    what = __fsub_rn(decayed, __fmul_rn(P.lr, u));
+    if (P.nesterov == 0u) {
+        const float u = __fdiv_rn(mh, den);
+        what = __fsub_rn(decayed, __fmul_rn(P.lr, u));
+    } else {
+        // NAdamW (Appendix B.1): gradient part and (uncorrected) momentum part over
+        // the same denominator, weighted by the momentum schedule's cg and cm
+        const float ug = __fdiv_rn(g, den);
+        const float um = __fdiv_rn(m, den);
+        what = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug)), __fmul_rn(P.cm, um));
+    }
 }
 
 template <int R>

@@ -43,7 +43,8 @@ def test_config_struct_matches_header_layout():
     assert offs["seed"] == 80 and offs["lookahead_delay"] == 88
     assert offs["device"] == 96 and offs["avg_interval"] == 100 and offs["stream"] == 104
     assert offs["alloc"] == 112 and offs["free"] == 120 and offs["alloc_ctx"] == 128
-    assert ctypes.sizeof(binding.Config) == 136
+    assert offs["optimizer"] == 136 and offs["pad0"] == 140 and offs["momentum_decay"] == 144
+    assert ctypes.sizeof(binding.Config) == 152
 
 
 def _cfg(**over):
@@ -64,7 +65,7 @@ def _cfg(**over):
     (dict(p=-0.1), "p ="), (dict(p=1.5), "p ="), (dict(p=float("nan")), "p ="),
     (dict(tau=65), "tau"), (dict(ema_beta=1.01), "ema_beta"), (dict(lr=0.0), "lr"),
     (dict(eps=0.0), "eps"), (dict(beta1=1.0), "betas"), (dict(tau=3, avg_interval=2), "avg_interval"),
-    (dict(avg_interval=-1), "avg_interval"), (dict(flags=8), "flags"),
+    (dict(avg_interval=-1), "avg_interval"), (dict(optimizer=2), "optimizer"), (dict(flags=8), "flags"),
 ])
 def test_create_rejects_bad_arguments_without_touching_a_device(lib, over, word):
     h = ctypes.c_void_p()
@@ -122,3 +123,20 @@ def test_product_does_not_import_the_oracle():
     for f in os.listdir(os.path.join(ROOT, "oracle")):
         if f.endswith((".py", ".c")):
             assert "paper_2601_22442_b200" not in open(os.path.join(ROOT, "oracle", f)).read()
+
+
+def test_paper_schedules():
+    from paper_2601_22442_b200 import ema_coefficient, learning_rate
+    T = 30000
+    # EMA coefficient: 0.5 for 1k iterations, then cosine to 0.01 (Section 3.3)
+    assert ema_coefficient(1, T) == 0.5 and ema_coefficient(1000, T) == 0.5
+    assert abs(ema_coefficient(T, T) - 0.01) < 1e-12
+    mid = 1000 + (T - 1000) // 2
+    assert abs(ema_coefficient(mid, T) - 0.255) < 1e-4
+    vals = [ema_coefficient(t, T) for t in range(1, T + 1, 97)]
+    assert all(a >= b for a, b in zip(vals, vals[1:])) and 0.01 <= min(vals)
+    # learning rate: linear warm-up 1e-7 -> 3e-4 over 3k, cosine to 3e-5 (Appendix B.1)
+    assert abs(learning_rate(3000, T) - 3e-4) < 1e-15
+    assert abs(learning_rate(1500, T) - (1e-7 + (3e-4 - 1e-7) / 2)) < 1e-15
+    assert abs(learning_rate(T, T) - 3e-5) < 1e-15
+    assert learning_rate(1, T) < 3e-7 and learning_rate(16500, T) == pytest.approx(1.65e-4, rel=1e-3)

@@ -26,11 +26,12 @@ def am():
 
 
 def make_pair(R, numel, p, tau, lam, delays=None, seed=0x5EED, hp=HP, same_init=True,
-              init_seed=0x1217, flags=0, avg_interval=1):
+              init_seed=0x1217, flags=0, avg_interval=1, optimizer="adamw"):
     o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
-                      lookahead_delay=delays, avg_interval=avg_interval, **hp)
+                      lookahead_delay=delays, avg_interval=avg_interval, optimizer=optimizer, **hp)
     g = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
-                       lookahead_delay=delays, flags=flags, avg_interval=avg_interval, **hp)
+                       lookahead_delay=delays, flags=flags, avg_interval=avg_interval,
+                       optimizer=optimizer, **hp)
     for s, n in enumerate(numel):
         if same_init:
             w0 = si.init_weights_host(init_seed, s, 0, n)
@@ -169,6 +170,16 @@ def test_averaging_interval(K, tau, p):
     from paper_2601_22442_b200 import binding
     run_case(4, [5000, 1024 * 2 + 3], p, tau, 0.9, steps=4 * K + tau + 1, avg_interval=K)
     run_case(3, [5000], p, tau, 0.9, steps=3 * K + tau + 1, avg_interval=K,
+             flags=binding.FLAG_DIRECT_KERNEL)
+
+
+@pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (2, 0.4)])
+def test_nadamw(tau, p):
+    # the paper's own optimizer for asynchronous pipelines (momentum 0.99)
+    from paper_2601_22442_b200 import binding
+    hp = dict(HP, beta1=0.99, weight_decay=0.01)
+    run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp)
+    run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
              flags=binding.FLAG_DIRECT_KERNEL)
 
 
