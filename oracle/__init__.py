@@ -54,6 +54,10 @@ def lib() -> ctypes.CDLL:
                                        dbl, dbl, dbl, u64, vp, u32]
         L.am_oracle_set_optimizer.restype = None
         L.am_oracle_set_optimizer.argtypes = [vp, u32, dbl]
+        L.am_oracle_set_exchange.restype = None
+        L.am_oracle_set_exchange.argtypes = [vp, u32]
+        L.am_oracle_exchanged.restype = ctypes.c_float
+        L.am_oracle_exchanged.argtypes = [u32, ctypes.c_float]
         L.am_oracle_destroy.restype = None
         L.am_oracle_destroy.argtypes = [vp]
         L.am_oracle_init_params.restype = ctypes.c_int
@@ -89,6 +93,11 @@ def philox4x32_10(ctr: Sequence[int], key: Sequence[int]) -> tuple:
     return tuple(int(x) for x in o)
 
 
+def exchanged(x: float, exchange: str = "bf16") -> float:
+    """A snapshot value as the other replicas see it (bf16: rounded to bfloat16)."""
+    return float(lib().am_oracle_exchanged({"fp32": 0, "bf16": 1}[exchange], float(x)))
+
+
 def threshold(p: float) -> int:
     return int(lib().am_oracle_threshold(float(p)))
 
@@ -115,7 +124,8 @@ class Oracle:
                  weight_decay: float = 0.1, seed: int = 0x5EED,
                  lookahead_delay: Optional[Sequence[int]] = None,
                  coord_base: Optional[Sequence[int]] = None, avg_interval: int = 1,
-                 optimizer: str = "adamw", momentum_decay: float = 4e-3):
+                 optimizer: str = "adamw", momentum_decay: float = 4e-3,
+                 exchange: str = "fp32"):
         self.R, self.S, self.tau = int(R), len(numel), int(tau)
         self.numel = [int(n) for n in numel]
         self.p, self.seed = float(p), int(seed)
@@ -132,6 +142,7 @@ class Oracle:
             raise ValueError("oracle: invalid configuration or out of memory")
         lib().am_oracle_set_optimizer(self._h, {"adamw": 0, "nadamw": 1}[optimizer],
                                       float(momentum_decay))
+        lib().am_oracle_set_exchange(self._h, {"fp32": 0, "bf16": 1}[exchange])
 
     def close(self) -> None:
         if getattr(self, "_h", None):

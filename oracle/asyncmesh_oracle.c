@@ -71,6 +71,7 @@ typedef struct am_oracle {
     uint32_t R, S, tau;
     uint32_t K;           /* averaging interval: subsets are exchanged at steps t = K, 2K, ... */
     uint32_t optimizer;   /* 0 AdamW, 1 NAdamW                                                  */
+    uint32_t exchange;    /* 0: subsets exchanged in fp32; 1: rounded to bfloat16 on the wire    */
     double momentum_decay, mu_product; /* NAdam's momentum schedule and its running product      */
     uint64_t *numel;      /* [S] coordinates held for stage j               */
     uint64_t *coord_base; /* [S] global index of local coordinate 0         */
@@ -212,6 +213,39 @@ int am_oracle_init_params(am_oracle *o, uint32_t stage, int32_t replica,
 /* ---- one step ------------------------------------------------------------ */
 
 /*
+ * What a replica's snapshot value looks like to the others.  The paper's
+ * quantisation study (Section 4 "robustness", Appendix B.2) sends the subset in
+ * reduced precision; with exchange = 1 every value entering the average is
+ * first rounded to bfloat16 (round to nearest even: keep the upper 16 bits of
+ * the binary32 pattern), the average itself is formed in fp32, and a replica's
+ * own staleness sample still uses its own unrounded value, which never left it.
+ */
+static float exchanged(const am_oracle *o, float x)
+{
+    if (o->exchange == 0) return x;
+    uint32_t u;
+    memcpy(&u, &x, sizeof u);
+    if ((u & 0x7F800000u) != 0x7F800000u)          /* finite: round to nearest even */
+        u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    memcpy(&x, &u, sizeof x);
+    return x;
+}
+
+void am_oracle_set_exchange(am_oracle *o, uint32_t exchange)
+{
+    if (o) o->exchange = exchange;
+}
+
+float am_oracle_exchanged(uint32_t exchange, float x)
+{
+    am_oracle tmp;
+    memset(&tmp, 0, sizeof tmp);
+    tmp.exchange = exchange;
+    return exchanged(&tmp, x);
+}
+
+/*
  * grads[j] points to [R][numel_j] floats, row i = gradient of replica i.
  * lambda_t / lr_t < 0 mean "use the constant given at creation"; otherwise
  * they replace it for this step (the paper decays both over training).
@@ -296,8 +330,9 @@ int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
                 sel = am_oracle_selected(o->seed, o->thresh, s, u_step,
                                          o->coord_base[s] + mu);
             if (sel) {
-                float a = Hold[mu];
-                for (uint32_t i = 1; i < R; ++i) a = a + Hold[(uint64_t)i * N + mu];
+                float a = exchanged(o, Hold[mu]);
+                for (uint32_t i = 1; i < R; ++i)
+                    a = a + exchanged(o, Hold[(uint64_t)i * N + mu]);
                 const float abar = a / Rf;
                 for (uint32_t i = 0; i < R; ++i) {
                     const uint64_t k = (uint64_t)i * N + mu;

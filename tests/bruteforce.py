@@ -30,8 +30,17 @@ def in_subset(seed, p, stage, step, mu):
     return x[mu & 3] < int(np.floor(p * 4294967296.0))
 
 
+def to_wire(ft, x, wire):
+    """A value as sent to the other replicas: unchanged, or rounded to bfloat16 by
+    the tensor library's own conversion."""
+    if wire == "fp32":
+        return x
+    import torch
+    return ft(torch.tensor(float(x), dtype=torch.float32).to(torch.bfloat16).to(torch.float32).item())
+
+
 def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
-        stage=0, interval=1):
+        stage=0, interval=1, wire="fp32"):
     """grads[t-1][i][mu] for t = 1..T.  Returns a list of per-step records."""
     T = len(grads)
     w = [[ft(w0[mu]) for mu in range(N)] for _ in range(R)]
@@ -66,9 +75,9 @@ def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
             # t - tau is consumed at round t
             if t % interval == 0 and t - tau >= 1 and mu in subsets[t - tau]:
                 old = hist[t - tau]
-                acc = old[0][mu]
+                acc = to_wire(ft, old[0][mu], wire)
                 for i in range(1, R):
-                    acc = ft(acc + old[i][mu])
+                    acc = ft(acc + to_wire(ft, old[i][mu], wire))
                 wbar = ft(acc / ft(R))
                 for i in range(R):
                     stal = ft(what[i][mu] - old[i][mu])

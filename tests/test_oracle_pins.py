@@ -407,6 +407,39 @@ def test_bruteforce_trace_with_averaging_interval(K, tau):
         oracle.Oracle(R, [N], p=0.5, tau=3, ema_beta=0.7, avg_interval=2)
 
 
+def test_bf16_rounding_against_the_tensor_library():
+    rng = np.random.default_rng(5)
+    xs = np.concatenate([
+        rng.standard_normal(20000).astype(np.float32) * 0.02,
+        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895314e38, 1e-40, -1e-40,
+                  1.0 + 2 ** -8, 1.0 + 3 * 2 ** -9], dtype=np.float32)])   # ties and edges
+    ref = torch.tensor(xs).to(torch.bfloat16).to(torch.float32).numpy()
+    got = np.array([oracle.exchanged(float(x)) for x in xs], dtype=np.float32)
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+    assert oracle.exchanged(0.1234567, "fp32") == float(np.float32(0.1234567))
+
+
+@pytest.mark.parametrize("tau", [0, 2])
+def test_bruteforce_trace_with_bf16_exchange(tau):
+    # the average is formed from bfloat16-rounded snapshots, the staleness sample
+    # from the replica's own unrounded value
+    R, N, T, seed = 3, 16, 8, 0x99
+    w0, grads = rand_setup(R, N, T, seed=31)
+    o = oracle.Oracle(R, [N], p=0.5, tau=tau, ema_beta=0.6, seed=seed, lookahead_delay=[1],
+                      exchange="bf16", **HP)
+    ref = oracle.Oracle(R, [N], p=0.5, tau=tau, ema_beta=0.6, seed=seed, lookahead_delay=[1], **HP)
+    o.init_params(0, w0); ref.init_params(0, w0)
+    args = (R, N, 0.5, tau, 0.6, HP["lr"], HP["beta1"], HP["beta2"], HP["eps"],
+            HP["weight_decay"], seed, 1, w0, grads)
+    tr = bruteforce.run(np.float32, *args, wire="bf16")
+    for t in range(1, T + 1):
+        o.step([grads[t - 1]]); ref.step([grads[t - 1]])
+        for name in ("w", "m", "v", "d", "look"):
+            assert (o.get(0, name).astype(np.float64) == tr[t - 1][name]).all(), (t, name)
+    diff = np.abs(o.get(0, "w") - ref.get(0, "w")).max()
+    assert 0 < diff < 1e-3        # it matters, by about a bfloat16 ulp of |w| ~ 0.05
+
+
 # ---- P9: elementwise independence ---------------------------------------------------
 
 def test_coordinate_slice_evolves_like_the_full_vector():
