@@ -57,6 +57,11 @@ extern "C" {
                                           where the shared-memory pipelined one applies  */
 #define ASYNCMESH_FLAG_PIPELINED_KERNEL 4u /* use the compact ring and the pipelined kernel for
                                              any p (diagnostic: exercises its in-place path) */
+#define ASYNCMESH_FLAG_BF16_EXCHANGE 16u /* the subset is exchanged in bfloat16 (the paper's
+                                           quantisation study): every snapshot value entering the
+                                           replica average is first rounded to bfloat16 (nearest
+                                           even); the average is formed in fp32 and a replica's own
+                                           staleness sample uses its own unrounded value         */
 
 /* state selectors of asyncmesh_read_state */
 #define ASYNCMESH_STATE_W 0     /* weights w_i^t                               */

@@ -21,6 +21,7 @@ ERR_BAD_STATE, ERR_UNSUPPORTED, ERR_DEVICE_STATUS = -4, -5, -6
 FLAG_SMALL_RING = 1
 FLAG_DIRECT_KERNEL = 2
 FLAG_PIPELINED_KERNEL = 4
+FLAG_BF16_EXCHANGE = 16
 STATE = {"w": 0, "m": 1, "v": 2, "d": 3, "look": 4}
 
 ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t)

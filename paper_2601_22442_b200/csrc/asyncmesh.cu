@@ -77,6 +77,7 @@ struct KernelChoice {
 
 struct asyncmesh {
     uint32_t R = 0, S = 0, tau = 0;
+    uint32_t wire_bf16 = 0;           // ASYNCMESH_FLAG_BF16_EXCHANGE
     uint32_t optimizer = 0;           // ASYNCMESH_OPT_*
     double momentum_decay = 4e-3, mu_product = 1.0;   // NAdamW's momentum schedule
     uint32_t K = 1;                   // averaging interval in steps; tau is a multiple of it
@@ -316,7 +317,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if (!(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: betas must lie in [0, 1)");
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
-                        ASYNCMESH_FLAG_PIPELINED_KERNEL)) != 0)
+                        ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
     if (cfg->optimizer > ASYNCMESH_OPT_NADAMW || cfg->pad0 != 0 || !(cfg->momentum_decay >= 0.0))
         return fail(ASYNCMESH_ERR_INVALID_ARG,
@@ -348,6 +349,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     h->R = cfg->R; h->S = cfg->S; h->tau = cfg->tau;
     h->K = K; h->lag = cfg->tau / K;
     h->optimizer = cfg->optimizer;
+    h->wire_bf16 = (cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) ? 1u : 0u;
     h->momentum_decay = cfg->momentum_decay > 0.0 ? cfg->momentum_decay : 4e-3;
     h->p = cfg->p; h->ema_beta = cfg->ema_beta; h->lr = cfg->lr;
     h->beta1 = cfg->beta1; h->beta2 = cfg->beta2; h->eps = cfg->eps; h->wd = cfg->weight_decay;
@@ -592,6 +594,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.lam = (float)lam;
     P.oml = (float)(1.0 - lam);
     P.Rf = (float)h->R;
+    P.wire_bf16 = h->wire_bf16;
     P.nesterov = h->optimizer == ASYNCMESH_OPT_NADAMW ? 1u : 0u;
     double mu_product = h->mu_product;
     if (P.nesterov) {   // mu_t, mu_{t+1} and the running product of the momentum schedule

@@ -31,6 +31,7 @@
 // result; the same operation order is what the CPU check uses.
 #pragma once
 #include <cstdint>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "philox.cuh"
@@ -76,6 +77,7 @@ struct StepParams {
     uint32_t prod_slot, cons_slot;
     SubsetRule rule;
     float b1, b2, omb1, omb2, ib1, ib2, eps, lr, lrwd, lam, oml, Rf;
+    uint32_t wire_bf16;          // snapshots enter the average rounded to bfloat16
     uint32_t nesterov;           // 0: AdamW, 1: NAdamW
     float cg, cm;                // NAdamW: weights of the gradient and momentum parts
 };
@@ -87,6 +89,15 @@ __device__ __forceinline__ float4 ld_stream(const float *p)
 __device__ __forceinline__ void st_stream(float *p, const float (&x)[4])
 {
     __stcs(reinterpret_cast<float4 *>(p), make_float4(x[0], x[1], x[2], x[3]));
+}
+
+// A snapshot value as the other replicas see it: unchanged, or rounded to
+// bfloat16 (round to nearest even) when the subset is exchanged in reduced
+// precision (the paper's quantisation study).  The average is formed in fp32; a
+// replica's own staleness sample keeps using its own unrounded value.
+__device__ __forceinline__ float on_wire(const StepParams &P, float x)
+{
+    return P.wire_bf16 ? __bfloat162float(__float2bfloat16_rn(x)) : x;
 }
 
 // The local optimizer step (first line of Eq. "sparta"), one rounding per written
@@ -224,9 +235,9 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                         ce[j] = idx * R;
                         float old[R];
                         load_replicas<R>(ring_cons + ce[j], old);
-                        float a = old[0];
+                        float a = on_wire(P, old[0]);
 #pragma unroll
-                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, old[i]);
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire(P, old[i]));
                         abar[j] = __fdiv_rn(a, P.Rf);
                     }
                 }
@@ -313,7 +324,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                 } else {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        acc[c] = (i == 0) ? wh[c] : __fadd_rn(acc[c], wh[c]);
+                        acc[c] = (i == 0) ? on_wire(P, wh[c]) : __fadd_rn(acc[c], on_wire(P, wh[c]));
                         wold_keep[i][c] = w[c];
                     }
                 }

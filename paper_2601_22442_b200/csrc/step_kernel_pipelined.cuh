@@ -378,9 +378,9 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                                 const uint64_t ce = (uint64_t)(cfirst + __popc(cm & below)) * R;
                                 float old[R];
                                 load_replicas<R>(ring_cons + ce, old);
-                                float a = old[0];
+                                float a = on_wire(P, old[0]);
 #pragma unroll
-                                for (int q = 1; q < R; ++q) a = __fadd_rn(a, old[q]);
+                                for (int q = 1; q < R; ++q) a = __fadd_rn(a, on_wire(P, old[q]));
                                 const float abar = __fdiv_rn(a, P.Rf);
                                 float *dp = st.D + (mu0 + (uint64_t)(j >> 2) * 128 + (j & 3)) * R + i;
                                 float old_i = old[0];
@@ -437,9 +437,9 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         // Eq. "ema" + corrected averaging on S^{t-tau}
                         float wold[R];
                         load_replicas<R>(st_wold + q * R, wold);
-                        float a = s_old[0];
+                        float a = on_wire(P, s_old[0]);
 #pragma unroll
-                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, s_old[i]);
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire(P, s_old[i]));
                         const float abar = __fdiv_rn(a, P.Rf);
 #pragma unroll
                         for (int i = 0; i < R; ++i) {

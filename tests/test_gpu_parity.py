@@ -26,9 +26,12 @@ def am():
 
 
 def make_pair(R, numel, p, tau, lam, delays=None, seed=0x5EED, hp=HP, same_init=True,
-              init_seed=0x1217, flags=0, avg_interval=1, optimizer="adamw"):
+              init_seed=0x1217, flags=0, avg_interval=1, optimizer="adamw", exchange="fp32"):
+    if exchange == "bf16":
+        flags |= 16
     o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
-                      lookahead_delay=delays, avg_interval=avg_interval, optimizer=optimizer, **hp)
+                      lookahead_delay=delays, avg_interval=avg_interval, optimizer=optimizer,
+                      exchange=exchange, **hp)
     g = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
                        lookahead_delay=delays, flags=flags, avg_interval=avg_interval,
                        optimizer=optimizer, **hp)
@@ -181,6 +184,22 @@ def test_nadamw(tau, p):
     run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp)
     run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
              flags=binding.FLAG_DIRECT_KERNEL)
+
+
+@pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (3, 0.4)])
+def test_bf16_exchange(tau, p):
+    # subsets exchanged in bfloat16: all three ring modes and both compact-ring kernels
+    from paper_2601_22442_b200 import binding
+    o, g = run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 5, exchange="bf16")
+    run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="bf16",
+             flags=binding.FLAG_DIRECT_KERNEL)
+    # and it is not the fp32 exchange
+    ref = oracle.Oracle(4, [6000, 1024 + 9], p=p, tau=tau, ema_beta=0.9, **HP)
+    for s, n in enumerate([6000, 1024 + 9]):
+        ref.init_params(s, si.init_weights_host(0x1217, s, 0, n))
+    for t in range(1, 3 * tau + 6):
+        ref.step([si.grads_host(0x6AD5, t, s, 4, 0, n) for s, n in enumerate([6000, 1024 + 9])])
+    assert np.abs(ref.get(0, "w") - g.get(0, "w")).max() > 0
 
 
 @pytest.mark.parametrize("lam", [0.0, 1.0])
