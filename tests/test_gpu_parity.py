@@ -318,6 +318,29 @@ def test_ring_overflow_is_reported_not_silent():
     h.status()
 
 
+def test_limits_of_the_interface():
+    # as many stages, replicas and steps of delay as the interface allows
+    sizes = [257 + 31 * k for k in range(64)]
+    run_case(2, sizes, 0.1, 1, 0.9, steps=4)
+    run_case(16, [3000, 1100], 0.05, 3, 0.9, steps=8)
+    o, g = run_case(2, [2100], 0.2, 64, 0.9, steps=70)
+    assert g.get(0, "d").any()
+    run_case(2, [2100], 1.0, 64, 0.5, steps=67)        # dense ring, 64 slots
+
+
+def test_gradient_buffers_are_not_modified_and_steps_are_stream_ordered():
+    g = am().AsyncMesh(2, [5000], p=0.3, tau=1, ema_beta=0.9, **HP)
+    g.init_params(0, si.init_weights_host(1, 0, 0, 5000))
+    bufs = g.empty_grads()
+    si.grads_device(bufs[0], 3, 1, 0, 5000)
+    before = bufs[0].clone()
+    for _ in range(5):
+        g.step(bufs)
+    g.status()
+    assert torch.equal(before, bufs[0])
+    assert g.min_bytes_last_step() == int((28 + 16 * 0.3) * 2 * 5000)
+
+
 def test_toy_config_100_steps():
     # the small benchmark configuration: R=4, S=2, 2^20 per stage, p=0.05, tau=1,
     # beta=0.9, AdamW lr 3e-4 (0.9, 0.95) wd 0.1, delay = S-1-stage, 100 steps
