@@ -51,6 +51,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--flags", type=int, default=0, help="asyncmesh_config.flags (diagnostic)")
     return ap.parse_args()
 
 
@@ -249,7 +250,7 @@ def run_native(args):
     mesh = pkg.AsyncMesh(R, numel, p=hp["p"], tau=tau, ema_beta=hp["ema_beta"], lr=hp["lr"],
                          beta1=hp["beta1"], beta2=hp["beta2"], eps=hp["eps"],
                          weight_decay=hp["weight_decay"], seed=MESH_SEED + rank, device=local,
-                         stream=stream.cuda_stream)
+                         stream=stream.cuda_stream, flags=args.flags)
     for s, n in enumerate(numel):
         tmp = torch.empty(n, dtype=torch.float32, device=dev)
         si.normal_device(tmp, si.stream_key(INIT_SEED + rank, si.KIND_INIT, 0, s, 0), 0, 0.02)

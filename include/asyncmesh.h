@@ -62,6 +62,9 @@ extern "C" {
                                            replica average is first rounded to bfloat16 (nearest
                                            even); the average is formed in fp32 and a replica's own
                                            staleness sample uses its own unrounded value         */
+#define ASYNCMESH_FLAG_DENSE_RING 32u /* keep the snapshot ring dense (one position per coordinate
+                                        and replica, tau slots) whatever p is: more memory and
+                                        some more traffic, no compaction work                   */
 
 /* state selectors of asyncmesh_read_state */
 #define ASYNCMESH_STATE_W 0     /* weights w_i^t                               */

@@ -317,7 +317,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if (!(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: betas must lie in [0, 1)");
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
-                        ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE)) != 0)
+                        ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE |
+                        ASYNCMESH_FLAG_DENSE_RING)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
     if (cfg->optimizer > ASYNCMESH_OPT_NADAMW || cfg->pad0 != 0 || !(cfg->momentum_decay >= 0.0))
         return fail(ASYNCMESH_ERR_INVALID_ARG,
@@ -397,6 +398,9 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
     h->total_chunks = (uint32_t)chunks;
     if (h->tau == 0) { h->mode = kSync; h->n_slots = 0; }
+    else if ((cfg->flags & ASYNCMESH_FLAG_DENSE_RING) && !(cfg->flags & ASYNCMESH_FLAG_SMALL_RING)) {
+        h->mode = kDense; h->n_slots = h->lag;
+    }
     else if (dense_total <= compact_total &&
              !(cfg->flags & (ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_PIPELINED_KERNEL))) {
         h->mode = kDense; h->n_slots = h->lag;
@@ -738,7 +742,7 @@ extern "C" int asyncmesh_read_state_range(asyncmesh *h, uint32_t stage, int whic
     case ASYNCMESH_STATE_M: row = d.M; break;
     case ASYNCMESH_STATE_V: row = d.V; break;
     case ASYNCMESH_STATE_LOOK: row = d.LOOK; break;
-    case ASYNCMESH_STATE_D: break;
+    case ASYNCMESH_STATE_D: if (h->mode == kDense) row = d.D; break;   // replica-major there
     default: return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: unknown selector %d", which);
     }
     if (row) {

@@ -19,10 +19,11 @@
 //            base in chunk_base[slot][chunk]; tau steps later the consumer finds
 //            the data through that table and recomputes membership and rank
 //            from Philox, so no index list is stored.  tau + 1 slots.
-//   dense    slot = [row_stride][R], coordinate mu at position mu; used when the
-//            subset is so large that compaction saves nothing.  tau slots; the
-//            consumer and producer of a step share a slot and a thread reads a
-//            position before it overwrites it.
+//   dense    slot = [R][row_stride], replica-major like w, coordinate mu at position
+//            mu; used when the subset is so large that compaction saves nothing
+//            (d is replica-major too in this mode).  tau slots; the consumer and
+//            producer of a step share a slot and a thread reads a position
+//            before it overwrites it.
 // With tau = 0 (synchronous sparse averaging, Eq. "sparta") there is no ring:
 // the average is formed from the registers of the lane that owns the coordinate.
 //
@@ -51,7 +52,7 @@ constexpr int kStatusRingOverflow = 1;
 
 struct StageDesc {
     float *W, *M, *V;       // [R][stride]
-    float *D;               // [stride][R]
+    float *D;               // [stride][R]; [R][stride] with the dense ring
     float *LOOK;            // [R][stride]; == W when delta == 0
     float *ring;            // [n_slots][slot_floats]
     uint32_t *chunk_base;   // [n_slots][n_chunks]           (compact only)
@@ -219,6 +220,91 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
         if (mu >= N) break;   // no warp-wide operation below this point
         const uint32_t pm = (pmask >> (4 * k)) & 0xFu;
         const uint32_t cm = (cmask >> (4 * k)) & 0xFu;
+
+        if constexpr (MODE == kDense) {
+            // Large subsets: the ring slot and d are replica-major like w, m, v, so the
+            // sparse quantities stream as float4 too.  A lane owns its four coordinates
+            // in every replica row, reads a ring position before it overwrites it, and
+            // writes whole float4: ring positions of unselected coordinates are never
+            // read by anyone, and d is rewritten with its old value there.
+            // The stale values of all replicas go out first and are summed only after
+            // the first group's dense loads have been issued: instructions issue in
+            // order, so a sum placed right behind its loads would hold back every
+            // load after it for a full memory round trip.
+            float4 r4[R];
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                r4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (cm) r4[i] = *reinterpret_cast<const float4 *>(ring_cons + (uint64_t)i * stride + mu);
+            }
+            float abar[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i0 = 0; i0 < R; i0 += RG) {
+                float4 w4[RG], g4[RG], m4[RG], v4[RG], d4[RG];
+#pragma unroll
+                for (int ii = 0; ii < RG; ++ii) {
+                    const uint64_t off = (uint64_t)(i0 + ii) * stride + mu;
+                    w4[ii] = ld_stream(st.W + off);
+                    g4[ii] = ld_stream(G + off);
+                    m4[ii] = ld_stream(st.M + off);
+                    v4[ii] = ld_stream(st.V + off);
+                    d4[ii] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (cm) d4[ii] = ld_stream(st.D + off);
+                }
+                if (i0 == 0 && cm) {   // stale average, replica order, one division
+                    float a[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int i = 0; i < R; ++i) {
+                        const float r[4] = {r4[i].x, r4[i].y, r4[i].z, r4[i].w};
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            a[c] = (i == 0) ? on_wire(P, r[c]) : __fadd_rn(a[c], on_wire(P, r[c]));
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) abar[c] = __fdiv_rn(a[c], P.Rf);
+                }
+#pragma unroll
+                for (int ii = 0; ii < RG; ++ii) {
+                    const uint64_t off = (uint64_t)(i0 + ii) * stride + mu;
+                    const float4 o4 = r4[i0 + ii];
+                    const float w[4] = {w4[ii].x, w4[ii].y, w4[ii].z, w4[ii].w};
+                    const float g[4] = {g4[ii].x, g4[ii].y, g4[ii].z, g4[ii].w};
+                    float m[4] = {m4[ii].x, m4[ii].y, m4[ii].z, m4[ii].w};
+                    float v[4] = {v4[ii].x, v4[ii].y, v4[ii].z, v4[ii].w};
+                    const float old[4] = {o4.x, o4.y, o4.z, o4.w};
+                    float dd[4] = {d4[ii].x, d4[ii].y, d4[ii].z, d4[ii].w};
+                    float wh[4], wn[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        adamw(P, w[c], g[c], m[c], v[c], wh[c]);
+                        wn[c] = wh[c];
+                    }
+                    st_stream(st.M + off, m);
+                    st_stream(st.V + off, v);
+                    if (cm) {   // Eq. "ema" + corrected averaging on S^{t-tau}
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            if ((cm >> c) & 1u) {
+                                const float diff = __fsub_rn(wh[c], old[c]);
+                                dd[c] = __fadd_rn(__fmul_rn(P.oml, dd[c]), __fmul_rn(P.lam, diff));
+                                wn[c] = __fadd_rn(abar[c], dd[c]);
+                            }
+                        }
+                        st_stream(st.D + off, dd);
+                    }
+                    if (pm) st_stream(ring_prod + off, wh);   // snapshot of the local iterate on S^t
+                    st_stream(st.W + off, wn);
+                    if (has_look) {
+                        float lk[4];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            lk[c] = __fadd_rn(wn[c], __fmul_rn(delta, __fsub_rn(wn[c], w[c])));
+                        st_stream(st.LOOK + off, lk);
+                    }
+                }
+            }
+            continue;
+        }
 
         // ---- stale average wbar^{t-tau} of the coordinates being consumed -----
         float abar[4] = {0.f, 0.f, 0.f, 0.f};
