@@ -415,13 +415,17 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                     }
                 }
 
-                st_stream(st.W + off, wn);
-                if (has_look) {   // Section 2.2: extrapolate the last update direction
-                    float lk[4];
+                // (synchronous mode with all four coordinates selected: the replica
+                // mean below writes these float4 in one go, nothing to store yet)
+                if (MODE != kSync || pm != 0xFu) {
+                    st_stream(st.W + off, wn);
+                    if (has_look) {   // Section 2.2: extrapolate the last update direction
+                        float lk[4];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        lk[c] = __fadd_rn(wn[c], __fmul_rn(delta, __fsub_rn(wn[c], w[c])));
-                    st_stream(st.LOOK + off, lk);
+                        for (int c = 0; c < 4; ++c)
+                            lk[c] = __fadd_rn(wn[c], __fmul_rn(delta, __fsub_rn(wn[c], w[c])));
+                        st_stream(st.LOOK + off, lk);
+                    }
                 }
             }
         }
@@ -430,7 +434,24 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
             // Eq. "sparta": coordinates of S^t take the replica mean.  The EMA
             // state stays exactly zero when tau = 0 (its sample is w^ - w^ = 0),
             // so the corrected value is mean + 0.
-            if (pm) {
+            if (pm == 0xFu) {   // whole float4 selected (always so at p = 1): vector stores
+                float wnew[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) wnew[c] = __fadd_rn(__fdiv_rn(acc[c], P.Rf), 0.0f);
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    const uint64_t off = (uint64_t)i * stride + mu;
+                    st_stream(st.W + off, wnew);
+                    if (has_look) {
+                        float lk[4];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            lk[c] = __fadd_rn(wnew[c],
+                                              __fmul_rn(delta, __fsub_rn(wnew[c], wold_keep[i][c])));
+                        st_stream(st.LOOK + off, lk);
+                    }
+                }
+            } else if (pm) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     if ((pm >> j) & 1u) {
