@@ -282,10 +282,7 @@ static bool stash_fits(double p)
 {
     const double q = 1.0 - (1.0 - p) * (1.0 - p);
     const double mean = kPipeSubCoords * q, sd = std::sqrt(kPipeSubCoords * q * (1.0 - q));
-#ifndef AM_STASH_SIGMAS
-#define AM_STASH_SIGMAS 4.0
-#endif
-    return mean + AM_STASH_SIGMAS * sd <= (double)PipeCfg<4>::kStash;
+    return mean + 4.0 * sd <= (double)PipeCfg<4>::kStash;
 }
 
 // ---------------------------------------------------------------------------
