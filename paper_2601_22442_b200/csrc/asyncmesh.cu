@@ -102,7 +102,7 @@ struct asyncmesh {
     double *scratch = nullptr;        // one double for reductions
 
     int mode = kSync;
-    bool pipelined = false;
+    int pipelined = 0;
     KernelChoice kernel;
     uint32_t n_slots = 0;
     uint32_t total_chunks = 0;
@@ -234,18 +234,23 @@ static int grid_for(uint64_t items, int threads)
 // ---------------------------------------------------------------------------
 
 template <int R>
-static KernelChoice pick_mode(int mode, bool pipelined, uint32_t S)
+static KernelChoice pick_mode(int mode, int pipelined, uint32_t S)
 {
     KernelChoice c;
     switch (mode) {
     case kSync: c.fn = asyncmesh_step_kernel<R, kSync>; break;
     case kDense: c.fn = asyncmesh_step_kernel<R, kDense>; break;
     default:
-        if (pipelined) {
-            c.fn = asyncmesh_step_kernel_pipelined<R, AM_PIPE_STAGES>;
+        if (pipelined == 1) {
+            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeWide>;
             c.threads = kPipeThreads;
             c.smem = (size_t)pipe_table_bytes(S) +
-                     (size_t)(kPipeThreads / 32) * PipeCfg<R>::warp_bytes(AM_PIPE_STAGES);
+                     (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeWide>::warp_bytes(kPipeStages);
+        } else if (pipelined == 2) {
+            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeNarrow>;
+            c.threads = kPipeThreads;
+            c.smem = (size_t)pipe_table_bytes(S) +
+                     (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeNarrow>::warp_bytes(kPipeStages);
         } else {
             c.fn = asyncmesh_step_kernel<R, kCompact>;
         }
@@ -253,7 +258,7 @@ static KernelChoice pick_mode(int mode, bool pipelined, uint32_t S)
     return c;
 }
 
-static KernelChoice pick_kernel(uint32_t R, int mode, bool pipelined, uint32_t S)
+static KernelChoice pick_kernel(uint32_t R, int mode, int pipelined, uint32_t S)
 {
     switch (R) {
     case 1: return pick_mode<1>(mode, pipelined, S);
@@ -277,12 +282,13 @@ static KernelChoice pick_kernel(uint32_t R, int mode, bool pipelined, uint32_t S
 }
 
 // The pipelined kernel stashes the selected coordinates of a sub-iteration
-// (union of two subsets); it pays off while they fit its stash.
+// (union of two subsets); a shape pays off while they fit its stash.
+template <class SH>
 static bool stash_fits(double p)
 {
     const double q = 1.0 - (1.0 - p) * (1.0 - p);
-    const double mean = kPipeSubCoords * q, sd = std::sqrt(kPipeSubCoords * q * (1.0 - q));
-    return mean + 4.0 * sd <= (double)PipeCfg<4>::kStash;
+    const double mean = SH::kSubCoords * q, sd = std::sqrt(SH::kSubCoords * q * (1.0 - q));
+    return mean + 4.0 * sd <= (double)SH::CAP;
 }
 
 // ---------------------------------------------------------------------------
@@ -398,15 +404,21 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     else if ((cfg->flags & ASYNCMESH_FLAG_DENSE_RING) && !(cfg->flags & ASYNCMESH_FLAG_SMALL_RING)) {
         h->mode = kDense; h->n_slots = h->lag;
     }
-    else if (dense_total <= compact_total &&
+    // dense once compaction would save less than a third of the ring: from there on
+    // nearly every coordinate is selected and streaming beats per-coordinate work
+    else if (dense_total <= 1.5L * compact_total &&
              !(cfg->flags & (ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_PIPELINED_KERNEL))) {
         h->mode = kDense; h->n_slots = h->lag;
     }
     else { h->mode = kCompact; h->n_slots = h->lag + 1; }
 
     // the compact ring has two kernels; which one is fixed for the handle's life
-    h->pipelined = h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
-                   (stash_fits(cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL));
+    h->pipelined = 0;   // 0 direct, 1 pipelined wide, 2 pipelined narrow
+    if (h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL)) {
+        if (stash_fits<PipeWide>(cfg->p)) h->pipelined = 1;
+        else if (stash_fits<PipeNarrow>(cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL))
+            h->pipelined = 2;
+    }
 
     auto bail = [&](int code, const char *what) {
         release_all(h);

@@ -24,31 +24,27 @@
 #pragma once
 #include "step_kernel.cuh"
 
-#ifndef AM_PIPE_STAGES
-#define AM_PIPE_STAGES 3      // units in the shared-memory ring of a warp
-#endif
-#ifndef AM_PIPE_MIN_BLOCKS
-#define AM_PIPE_MIN_BLOCKS 2  // blocks per SM the register budget is sized for
-#endif
-#ifndef AM_PIPE_WIDTH
-#define AM_PIPE_WIDTH 2       // float4 per lane, array and unit (V)
-#endif
-#ifndef AM_PIPE_STASH
-#define AM_PIPE_STASH 64      // selected coordinates a sub-iteration can stash
-#endif
-#ifndef AM_PIPE_THREADS
-#define AM_PIPE_THREADS 192
-#endif
-
 namespace amk {
 
-constexpr int kPipeV = AM_PIPE_WIDTH;
-constexpr int kPipeThreads = AM_PIPE_THREADS;
-constexpr int kPipeSubCoords = 128 * kPipeV;            // coordinates per sub-iteration
-constexpr int kPipeSubIters = kWarpChunk / kPipeSubCoords;
-constexpr int kPipeBits = 4 * kPipeV;                   // mask bits per lane and sub-iteration
-constexpr int kUnitBytes = 4 * kPipeV * 512;            // w, g, m, v: V float4 per lane each
-static_assert(kPipeSubIters * kPipeBits == 32, "a lane's chunk mask must fill 32 bits");
+constexpr int kPipeThreads = 192;   // 6 warps; 2 blocks per SM
+constexpr int kPipeStages = 3;      // units in the shared-memory ring of a warp
+
+// Two shapes of the same kernel.  Wide: 8 coordinates per lane and unit, stash
+// for 64 selected coordinates per 256: the small subsets the paper works with.
+// Narrow: 4 coordinates per lane and unit, stash for all 128 coordinates of a
+// sub-iteration: any larger subset (until the dense ring takes over).
+template <int V_, int CAP_>
+struct PipeShape {
+    static constexpr int V = V_;                        // float4 per lane, array and unit
+    static constexpr int CAP = CAP_;                    // selected coordinates a sub-iteration can stash
+    static constexpr int kSubCoords = 128 * V;          // coordinates per sub-iteration
+    static constexpr int kSubIters = kWarpChunk / kSubCoords;
+    static constexpr int kBits = 4 * V;                 // mask bits per lane and sub-iteration
+    static constexpr int kUnitBytes = 4 * V * 512;      // w, g, m, v: V float4 per lane each
+    static_assert(kSubIters * kBits == 32, "a lane's chunk mask must fill 32 bits");
+};
+using PipeWide = PipeShape<2, 64>;
+using PipeNarrow = PipeShape<1, 128>;
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr)
 {
@@ -87,14 +83,14 @@ __device__ __forceinline__ void store_replicas(float *p, const float (&x)[R])
     }
 }
 
-template <int R>
+template <int R, class SH>
 struct PipeCfg {
-    static constexpr int kStash = AM_PIPE_STASH;
+    static constexpr int kStash = SH::CAP;
     static constexpr int kStashWords = kStash * (2 * R + 3);   // what, wold, coord, cidx, pidx
     static constexpr int kStashBytes = (kStashWords * 4 + 15) / 16 * 16;
     __host__ __device__ static constexpr int warp_bytes(int stages)
     {
-        return stages * kUnitBytes + kStashBytes;
+        return stages * SH::kUnitBytes + kStashBytes;
     }
 };
 
@@ -104,11 +100,12 @@ __host__ __device__ constexpr int pipe_table_bytes(uint32_t S)
     return (int)((S * sizeof(StageDesc) + 15) / 16 * 16);
 }
 
+template <class SH>
 __device__ __forceinline__ int pipe_sub_iterations(uint64_t N, uint32_t chunk)
 {
     const uint64_t rem = N - (uint64_t)chunk * kWarpChunk;
-    return rem >= (uint64_t)kWarpChunk ? kPipeSubIters
-                                       : (int)((rem + kPipeSubCoords - 1) / kPipeSubCoords);
+    return rem >= (uint64_t)kWarpChunk ? SH::kSubIters
+                                       : (int)((rem + SH::kSubCoords - 1) / SH::kSubCoords);
 }
 
 // Walks the warp's units in the order the arithmetic consumes them (chunk by
@@ -123,6 +120,7 @@ struct UnitCursor {
     bool valid;
 };
 
+template <class SH>
 __device__ __forceinline__ void cursor_enter_chunk(UnitCursor &c, const StepParams &P,
                                                    const StageDesc *sd, int lane)
 {
@@ -133,49 +131,51 @@ __device__ __forceinline__ void cursor_enter_chunk(UnitCursor &c, const StepPara
     const uint32_t chunk = c.gc - st.chunk_begin;
     c.W = st.W; c.M = st.M; c.V = st.V; c.G = P.G[c.s];
     c.N = st.N; c.stride = st.stride;
-    c.kmax = pipe_sub_iterations(st.N, chunk);
+    c.kmax = pipe_sub_iterations<SH>(st.N, chunk);
     c.k = 0;
     c.i = 0;
     c.mu0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
 }
 
-template <int R>
+template <int R, class SH>
 __device__ __forceinline__ void issue_unit(UnitCursor &c, const StepParams &P, const StageDesc *sd,
                                            uint32_t slot_addr, int lane, uint32_t n_warps)
 {
     if (c.valid) {
         const uint32_t a = slot_addr + lane * 16;
 #pragma unroll
-        for (int h = 0; h < kPipeV; ++h) {
+        for (int h = 0; h < SH::V; ++h) {
             const uint64_t mu = c.mu0 + (uint64_t)h * 128;
             if (mu < c.N) {
                 const uint64_t off = (uint64_t)c.i * c.stride + mu;
-                cp_async16(a + (0 * kPipeV + h) * 512, c.W + off);
-                cp_async16(a + (1 * kPipeV + h) * 512, c.G + off);
-                cp_async16(a + (2 * kPipeV + h) * 512, c.M + off);
-                cp_async16(a + (3 * kPipeV + h) * 512, c.V + off);
+                cp_async16(a + (0 * SH::V + h) * 512, c.W + off);
+                cp_async16(a + (1 * SH::V + h) * 512, c.G + off);
+                cp_async16(a + (2 * SH::V + h) * 512, c.M + off);
+                cp_async16(a + (3 * SH::V + h) * 512, c.V + off);
             }
         }
         if (++c.i == R) {
             c.i = 0;
-            c.mu0 += kPipeSubCoords;
+            c.mu0 += SH::kSubCoords;
             if (++c.k == c.kmax) {
                 c.gc += n_warps;
-                cursor_enter_chunk(c, P, sd, lane);
+                cursor_enter_chunk<SH>(c, P, sd, lane);
             }
         }
     }
     cp_async_commit();   // always: keeps the group count in step with the unit count
 }
 
-template <int R, int NST>
-__global__ void __launch_bounds__(kPipeThreads, AM_PIPE_MIN_BLOCKS)
+template <int R, int NST, class SH>
+__global__ void __launch_bounds__(kPipeThreads, 2)
 asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 {
-    using Cfg = PipeCfg<R>;
+    using Cfg = PipeCfg<R, SH>;
     constexpr int CAP = Cfg::kStash;
-    constexpr int V = kPipeV;
-    constexpr int NB = kPipeBits;   // mask bits per lane and sub-iteration
+    constexpr int V = SH::V;
+    constexpr int NB = SH::kBits;   // mask bits per lane and sub-iteration
+    constexpr int kUnitBytes = SH::kUnitBytes;
+    constexpr int kPipeSubCoords = SH::kSubCoords;
     extern __shared__ __align__(16) unsigned char dyn_smem_all[];
     StageDesc *sd = reinterpret_cast<StageDesc *>(dyn_smem_all);
     unsigned char *dyn_smem = dyn_smem_all + pipe_table_bytes(P.S);
@@ -205,10 +205,10 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
     UnitCursor pf;
     pf.gc = blockIdx.x * wpb + warp;
     pf.s = 0;
-    cursor_enter_chunk(pf, P, sd, lane);
+    cursor_enter_chunk<SH>(pf, P, sd, lane);
 #pragma unroll
     for (int q = 0; q < NST - 1; ++q)
-        issue_unit<R>(pf, P, sd, stage_base + q * kUnitBytes, lane, n_warps);
+        issue_unit<R, SH>(pf, P, sd, stage_base + q * kUnitBytes, lane, n_warps);
     uint32_t rd = 0, wr = NST - 1;   // ring slot being consumed / being filled
 
     const bool consume = P.consume != 0u;
@@ -219,7 +219,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         const uint32_t chunk = gc - st.chunk_begin;
         const uint64_t N = st.N, stride = st.stride;
         const uint64_t c0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
-        const int kmax = pipe_sub_iterations(N, chunk);
+        const int kmax = pipe_sub_iterations<SH>(N, chunk);
 
         // position of this chunk in the consumed slot and the membership mask stored
         // when that slot was produced: ask early, use late
@@ -331,7 +331,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 #pragma unroll(R <= 4 ? R : 1)
             for (int i = 0; i < R; ++i) {
                 cp_async_wait<NST - 2>();
-                issue_unit<R>(pf, P, sd, stage_base + wr * kUnitBytes, lane, n_warps);
+                issue_unit<R, SH>(pf, P, sd, stage_base + wr * kUnitBytes, lane, n_warps);
                 const unsigned char *slot = my + rd * kUnitBytes + lane * 16;
                 rd = (rd + 1 == NST) ? 0 : rd + 1;
                 wr = (wr + 1 == NST) ? 0 : wr + 1;
