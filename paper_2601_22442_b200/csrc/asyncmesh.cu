@@ -238,16 +238,25 @@ static KernelChoice pick_mode(int mode, int pipelined, uint32_t S)
 {
     KernelChoice c;
     switch (mode) {
-    case kSync: c.fn = asyncmesh_step_kernel<R, kSync>; break;
+    case kSync:
+        if (pipelined == 3) {
+            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeNarrow, kSync>;
+            c.threads = kPipeThreads;
+            c.smem = (size_t)pipe_table_bytes(S) +
+                     (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeNarrow>::warp_bytes(kPipeStages);
+        } else {
+            c.fn = asyncmesh_step_kernel<R, kSync>;
+        }
+        break;
     case kDense: c.fn = asyncmesh_step_kernel<R, kDense>; break;
     default:
         if (pipelined == 1) {
-            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeWide>;
+            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeWide, kCompact>;
             c.threads = kPipeThreads;
             c.smem = (size_t)pipe_table_bytes(S) +
                      (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeWide>::warp_bytes(kPipeStages);
         } else if (pipelined == 2) {
-            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeNarrow>;
+            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeNarrow, kCompact>;
             c.threads = kPipeThreads;
             c.smem = (size_t)pipe_table_bytes(S) +
                      (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeNarrow>::warp_bytes(kPipeStages);
@@ -413,7 +422,12 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     else { h->mode = kCompact; h->n_slots = h->lag + 1; }
 
     // the compact ring has two kernels; which one is fixed for the handle's life
-    h->pipelined = 0;   // 0 direct, 1 pipelined wide, 2 pipelined narrow
+    h->pipelined = 0;   // 0 direct, 1 pipelined wide, 2 pipelined narrow, 3 pipelined narrow synchronous
+    // synchronous mode: the stash route pays while most float4 groups are only partly
+    // selected; towards p = 1 the direct kernel writes whole groups and wins
+    if (h->mode == kSync && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
+        (cfg->p <= 0.8 || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL)))
+        h->pipelined = 3;
     if (h->mode == kCompact && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL)) {
         if (stash_fits<PipeWide>(cfg->p)) h->pipelined = 1;
         else if (stash_fits<PipeNarrow>(cfg->p) || (cfg->flags & ASYNCMESH_FLAG_PIPELINED_KERNEL))

@@ -166,10 +166,15 @@ __device__ __forceinline__ void issue_unit(UnitCursor &c, const StepParams &P, c
     cp_async_commit();   // always: keeps the group count in step with the unit count
 }
 
-template <int R, int NST, class SH>
+// MODE is kCompact (tau >= 1: ring, d, bitmap) or kSync (tau = 0, Eq. "sparta": the
+// replica mean of the selected coordinates is formed from the stash itself; needs
+// a stash that holds a whole sub-iteration, i.e. the narrow shape).
+template <int R, int NST, class SH, int MODE>
 __global__ void __launch_bounds__(kPipeThreads, 2)
 asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 {
+    static_assert(MODE == kCompact || (MODE == kSync && SH::CAP >= SH::kSubCoords),
+                  "the synchronous mode cannot fall back to in-place work");
     using Cfg = PipeCfg<R, SH>;
     constexpr int CAP = Cfg::kStash;
     constexpr int V = SH::V;
@@ -211,7 +216,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         issue_unit<R, SH>(pf, P, sd, stage_base + q * kUnitBytes, lane, n_warps);
     uint32_t rd = 0, wr = NST - 1;   // ring slot being consumed / being filled
 
-    const bool consume = P.consume != 0u;
+    const bool consume = (MODE == kCompact) && P.consume != 0u;
     uint32_t s = 0;
     for (uint32_t gc = blockIdx.x * wpb + warp; gc < P.total_chunks; gc += n_warps) {
         while (s + 1 < P.S && gc >= sd[s + 1].chunk_begin) ++s;
@@ -247,8 +252,10 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         }
 
         // ---- room in the producing slot -----------------------------------------
-        uint32_t pbase = 0, cexcl = 0, total;
-        const uint32_t pexcl = warp_exclusive_sum(__popc(pmask), lane, total);
+        uint32_t pbase = 0, cexcl = 0, pexcl = 0;
+        if constexpr (MODE == kCompact) {
+        uint32_t total;
+        pexcl = warp_exclusive_sum(__popc(pmask), lane, total);
         if (lane == 0) {
             uint32_t b = 0;
             if (total) {
@@ -270,6 +277,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         if (pbase == kInvalidBase) pmask = 0;
         if (P.produce)   // kept for step t + tau
             st.bitmap[(uint64_t)P.prod_slot * st.n_chunks * 32 + word] = pmask;
+        }
         const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
         float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
         const float delta = st.delta;
@@ -433,7 +441,23 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     }
                     float wh[R];
                     load_replicas<R>(st_what + q * R, wh);
-                    if (e_c != kInvalidBase) {
+                    if constexpr (MODE == kSync) {
+                        // Eq. "sparta": the selected coordinate takes the replica mean; the
+                        // EMA state stays exactly zero (its sample is w^ - w^), hence mean + 0
+                        float wold[R];
+                        load_replicas<R>(st_wold + q * R, wold);
+                        float a = on_wire(P, wh[0]);
+#pragma unroll
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire(P, wh[i]));
+                        const float wnew = __fadd_rn(__fdiv_rn(a, P.Rf), 0.0f);
+#pragma unroll
+                        for (int i = 0; i < R; ++i) {
+                            const uint64_t o1 = (uint64_t)i * stride + e_coord;
+                            st.W[o1] = wnew;
+                            if (has_look)
+                                st.LOOK[o1] = __fadd_rn(wnew, __fmul_rn(delta, __fsub_rn(wnew, wold[i])));
+                        }
+                    } else if (e_c != kInvalidBase) {
                         // Eq. "ema" + corrected averaging on S^{t-tau}
                         float wold[R];
                         load_replicas<R>(st_wold + q * R, wold);
@@ -454,7 +478,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         }
                         store_replicas<R>(st.D + (uint64_t)e_coord * R, s_dd);
                     }
-                    if (e_p != kInvalidBase)   // snapshot of the local iterate on S^t
+                    if (MODE == kCompact && e_p != kInvalidBase)   // snapshot of the local iterate on S^t
                         store_replicas<R>(ring_prod + (uint64_t)e_p * R, wh);
                 }
             }

@@ -141,6 +141,16 @@ def test_modes_small(tau, p):
     run_case(4, [5000, 3 * 1024 + 17], p, tau, 0.9, steps=3 * tau + 4)
 
 
+@pytest.mark.parametrize("flag", ["direct", "pipelined"])
+@pytest.mark.parametrize("R,p", [(4, 0.05), (8, 0.3), (3, 0.7), (2, 1.0), (5, 0.0)])
+def test_both_synchronous_kernels(flag, R, p):
+    # tau = 0 (Eq. "sparta") through the direct kernel and through the stash route
+    from paper_2601_22442_b200 import binding
+    f = binding.FLAG_DIRECT_KERNEL if flag == "direct" else binding.FLAG_PIPELINED_KERNEL
+    run_case(R, [9000, 1024 * 3 + 5, 77], p, 0, 0.9, steps=5, flags=f)
+    run_case(R, [5000], p, 0, 0.9, steps=6, flags=f, avg_interval=2, exchange="bf16")
+
+
 @pytest.mark.parametrize("R", [1, 2, 3, 5, 7, 8, 12, 16])
 def test_replica_counts(R):
     run_case(R, [2500], 0.3, 2, 0.9, steps=7)
