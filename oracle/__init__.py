@@ -56,6 +56,10 @@ def lib() -> ctypes.CDLL:
         L.am_oracle_set_optimizer.argtypes = [vp, u32, dbl]
         L.am_oracle_set_exchange.restype = None
         L.am_oracle_set_exchange.argtypes = [vp, u32]
+        L.am_oracle_set_correction.restype = None
+        L.am_oracle_set_correction.argtypes = [vp, u32]
+        L.am_oracle_ema_variance.restype = ctypes.c_int
+        L.am_oracle_ema_variance.argtypes = [vp, u32, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
         L.am_oracle_exchanged.restype = ctypes.c_float
         L.am_oracle_exchanged.argtypes = [u32, ctypes.c_float]
         L.am_oracle_destroy.restype = None
@@ -93,9 +97,13 @@ def philox4x32_10(ctr: Sequence[int], key: Sequence[int]) -> tuple:
     return tuple(int(x) for x in o)
 
 
+EXCHANGE = {"fp32": 0, "bf16": 1, "fp8": 2}
+CORRECTION = {"ema": 0, "eager": 1}
+
+
 def exchanged(x: float, exchange: str = "bf16") -> float:
-    """A snapshot value as the other replicas see it (bf16: rounded to bfloat16)."""
-    return float(lib().am_oracle_exchanged({"fp32": 0, "bf16": 1}[exchange], float(x)))
+    """A snapshot value as the other replicas see it (bf16 / fp8: rounded to that format)."""
+    return float(lib().am_oracle_exchanged(EXCHANGE[exchange], float(x)))
 
 
 def threshold(p: float) -> int:
@@ -125,7 +133,7 @@ class Oracle:
                  lookahead_delay: Optional[Sequence[int]] = None,
                  coord_base: Optional[Sequence[int]] = None, avg_interval: int = 1,
                  optimizer: str = "adamw", momentum_decay: float = 4e-3,
-                 exchange: str = "fp32"):
+                 exchange: str = "fp32", correction: str = "ema"):
         self.R, self.S, self.tau = int(R), len(numel), int(tau)
         self.numel = [int(n) for n in numel]
         self.p, self.seed = float(p), int(seed)
@@ -142,7 +150,8 @@ class Oracle:
             raise ValueError("oracle: invalid configuration or out of memory")
         lib().am_oracle_set_optimizer(self._h, {"adamw": 0, "nadamw": 1}[optimizer],
                                       float(momentum_decay))
-        lib().am_oracle_set_exchange(self._h, {"fp32": 0, "bf16": 1}[exchange])
+        lib().am_oracle_set_exchange(self._h, EXCHANGE[exchange])
+        lib().am_oracle_set_correction(self._h, CORRECTION[correction])
 
     def close(self) -> None:
         if getattr(self, "_h", None):
@@ -190,6 +199,13 @@ class Oracle:
 
     def consensus_error(self, stage: int) -> float:
         return float(lib().am_oracle_consensus_error(self._h, stage))
+
+    def ema_variance(self, stage: int) -> tuple:
+        """(mean, max) over the stage's coordinates of the across-replica variance of d."""
+        mean, mx = ctypes.c_double(), ctypes.c_double()
+        if lib().am_oracle_ema_variance(self._h, stage, ctypes.byref(mean), ctypes.byref(mx)) != 0:
+            raise ValueError("oracle: bad ema_variance request")
+        return float(mean.value), float(mx.value)
 
     def subset_mask(self, stage: int, step: int) -> np.ndarray:
         out = np.empty(self.numel[stage], dtype=np.uint8)

@@ -38,6 +38,11 @@
  *       steps") O3 runs only at steps t = K, 2K, ...; the steps in between are
  *       purely local (w^t = w^).  tau is then a multiple of K, so the average
  *       consumed at a round was launched at an earlier round.
+ *       The same paragraph names a second staleness estimate, that of eager
+ *       DiLoCo, as a special case (all parameters, tau = K):
+ *           d_i = (1/R) (w^_i^t[mu] - w^_i^{t-tau}[mu])
+ *       selectable here for any p, tau, K (correction = 1); w_i^t = wbar + d_i
+ *       as before.
  *   O4  pipeline look-ahead (Section 2.2): the last update direction
  *       (w^t - w^{t-1}) extrapolated by the stage's delay delta_j:
  *           look_i = w_i^t + delta_j (w_i^t - w_i^{t-1}).
@@ -71,7 +76,10 @@ typedef struct am_oracle {
     uint32_t R, S, tau;
     uint32_t K;           /* averaging interval: subsets are exchanged at steps t = K, 2K, ... */
     uint32_t optimizer;   /* 0 AdamW, 1 NAdamW                                                  */
-    uint32_t exchange;    /* 0: subsets exchanged in fp32; 1: rounded to bfloat16 on the wire    */
+    uint32_t exchange;    /* 0: subsets exchanged in fp32; 1: rounded to bfloat16 on the wire;
+                             2: rounded to 8-bit floating point (E4M3)                           */
+    uint32_t correction;  /* 0: EMA staleness estimate (Eq. "ema"); 1: eager estimate
+                             d_i = (w^_i^t - w^_i^{t-tau}) / R (end of Section 3.2)              */
     double momentum_decay, mu_product; /* NAdam's momentum schedule and its running product      */
     uint64_t *numel;      /* [S] coordinates held for stage j               */
     uint64_t *coord_base; /* [S] global index of local coordinate 0         */
@@ -217,12 +225,35 @@ int am_oracle_init_params(am_oracle *o, uint32_t stage, int32_t replica,
  * quantisation study (Section 4 "robustness", Appendix B.2) sends the subset in
  * reduced precision; with exchange = 1 every value entering the average is
  * first rounded to bfloat16 (round to nearest even: keep the upper 16 bits of
- * the binary32 pattern), the average itself is formed in fp32, and a replica's
- * own staleness sample still uses its own unrounded value, which never left it.
+ * the binary32 pattern), with exchange = 2 to 8-bit floating point (E4M3, the
+ * paper does not say which 8-bit format or scaling it used: plain cast, no
+ * scale); the average itself is formed in fp32, and a replica's own staleness
+ * sample still uses its own unrounded value, which never left it.
  */
+/*
+ * Nearest value of the 8-bit floating-point format E4M3 (4 exponent bits, bias 7,
+ * 3 mantissa bits, no infinities, largest finite value 448): ties to even,
+ * magnitudes above 448 clamp to 448, the spacing below 2^-6 is 2^-9 (subnormals).
+ */
+static float round_e4m3(float x)
+{
+    if (isnan(x)) return x;
+    float a = fabsf(x);
+    if (a > 448.0f) a = 448.0f;
+    if (a == 0.0f) return x;
+    int e;
+    (void)frexpf(a, &e);              /* a = f * 2^e with f in [0.5, 1): binade exponent e - 1 */
+    int q = (e - 1) - 3;              /* exponent of the spacing: three mantissa bits         */
+    if (q < -9) q = -9;               /* subnormal range                                      */
+    float r = ldexpf(nearbyintf(ldexpf(a, -q)), q);   /* nearbyintf: ties to even             */
+    if (r > 448.0f) r = 448.0f;
+    return copysignf(r, x);
+}
+
 static float exchanged(const am_oracle *o, float x)
 {
     if (o->exchange == 0) return x;
+    if (o->exchange == 2) return round_e4m3(x);
     uint32_t u;
     memcpy(&u, &x, sizeof u);
     if ((u & 0x7F800000u) != 0x7F800000u)          /* finite: round to nearest even */
@@ -235,6 +266,11 @@ static float exchanged(const am_oracle *o, float x)
 void am_oracle_set_exchange(am_oracle *o, uint32_t exchange)
 {
     if (o) o->exchange = exchange;
+}
+
+void am_oracle_set_correction(am_oracle *o, uint32_t correction)
+{
+    if (o) o->correction = correction;
 }
 
 float am_oracle_exchanged(uint32_t exchange, float x)
@@ -337,7 +373,11 @@ int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
                 for (uint32_t i = 0; i < R; ++i) {
                     const uint64_t k = (uint64_t)i * N + mu;
                     const float diff = what[k] - Hold[k];
-                    const float dk = (oml * d[k]) + (lam * diff);
+                    float dk;
+                    if (o->correction == 0)
+                        dk = (oml * d[k]) + (lam * diff);   /* Eq. "ema"          */
+                    else
+                        dk = diff / Rf;                     /* eager estimate     */
                     d[k] = dk;
                     w[k] = abar + dk;
                 }
@@ -416,6 +456,36 @@ double am_oracle_consensus_error(const am_oracle *o, uint32_t stage)
         }
     }
     return acc;
+}
+
+/* Spread of the staleness estimates across replicas (the appendix figure on the
+ * consensus error plots the "variance between EMA estimates in each replica",
+ * mean and max across the model dimension): per coordinate the population
+ * variance (1/R) sum_i (d_i - dbar)^2 in double; *mean_out = its mean over the
+ * stage's coordinates, *max_out = its maximum. */
+int am_oracle_ema_variance(const am_oracle *o, uint32_t stage, double *mean_out,
+                           double *max_out)
+{
+    if (!o || stage >= o->S || !mean_out || !max_out) return -1;
+    const uint64_t N = o->numel[stage];
+    double sum = 0.0, mx = 0.0;
+    for (uint64_t mu = 0; mu < N; ++mu) {
+        double mean = 0.0;
+        for (uint32_t i = 0; i < o->R; ++i)
+            mean += (double)o->d[stage][(uint64_t)i * N + mu];
+        mean /= (double)o->R;
+        double var = 0.0;
+        for (uint32_t i = 0; i < o->R; ++i) {
+            const double e = (double)o->d[stage][(uint64_t)i * N + mu] - mean;
+            var += e * e;
+        }
+        var /= (double)o->R;
+        sum += var;
+        if (var > mx) mx = var;
+    }
+    *mean_out = sum / (double)N;
+    *max_out = mx;
+    return 0;
 }
 
 /* One byte (0/1) per local coordinate: membership in S_stage^u. */

@@ -31,16 +31,17 @@ def in_subset(seed, p, stage, step, mu):
 
 
 def to_wire(ft, x, wire):
-    """A value as sent to the other replicas: unchanged, or rounded to bfloat16 by
-    the tensor library's own conversion."""
+    """A value as sent to the other replicas: unchanged, or rounded to bfloat16 / to
+    8-bit floating point (E4M3) by the tensor library's own conversion."""
     if wire == "fp32":
         return x
     import torch
-    return ft(torch.tensor(float(x), dtype=torch.float32).to(torch.bfloat16).to(torch.float32).item())
+    low = {"bf16": torch.bfloat16, "fp8": torch.float8_e4m3fn}[wire]
+    return ft(torch.tensor(float(x), dtype=torch.float32).to(low).to(torch.float32).item())
 
 
 def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
-        stage=0, interval=1, wire="fp32"):
+        stage=0, interval=1, wire="fp32", correction="ema"):
     """grads[t-1][i][mu] for t = 1..T.  Returns a list of per-step records."""
     T = len(grads)
     w = [[ft(w0[mu]) for mu in range(N)] for _ in range(R)]
@@ -81,7 +82,10 @@ def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
                 wbar = ft(acc / ft(R))
                 for i in range(R):
                     stal = ft(what[i][mu] - old[i][mu])
-                    d[i][mu] = ft(ft(oml * d[i][mu]) + ft(lamf * stal))
+                    if correction == "ema":      # Eq. "ema"
+                        d[i][mu] = ft(ft(oml * d[i][mu]) + ft(lamf * stal))
+                    else:                        # eager estimate, end of Section 3.2
+                        d[i][mu] = ft(stal / ft(R))
                     w[i][mu] = ft(wbar + d[i][mu])
             else:
                 for i in range(R):

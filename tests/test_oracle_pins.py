@@ -440,6 +440,129 @@ def test_bruteforce_trace_with_bf16_exchange(tau):
     assert 0 < diff < 1e-3        # it matters, by about a bfloat16 ulp of |w| ~ 0.05
 
 
+def e4m3_grid():
+    """All finite non-negative E4M3 values from the format's definition: bias 7, three
+    mantissa bits, subnormals at exponent field 0, top code of the top binade unused."""
+    vals = []
+    for e in range(16):
+        for mant in range(8):
+            if e == 15 and mant == 7:
+                continue                      # the NaN code
+            vals.append(mant / 8 * 2.0 ** -6 if e == 0 else (1 + mant / 8) * 2.0 ** (e - 7))
+    return vals
+
+
+def test_fp8_rounding_against_the_format_and_the_tensor_library():
+    grid = e4m3_grid()
+    assert grid[-1] == 448.0 and grid[1] == 2.0 ** -9 and len(grid) == 127
+    for k, x in enumerate(grid):              # representable values are fixed points
+        assert oracle.exchanged(x, "fp8") == x and oracle.exchanged(-x, "fp8") == -x
+        if k + 1 < len(grid):                 # the midpoint goes to the even code
+            mid = (x + grid[k + 1]) / 2
+            want = x if k % 2 == 0 else grid[k + 1]
+            assert oracle.exchanged(mid, "fp8") == want, (x, grid[k + 1])
+            assert oracle.exchanged(float(np.nextafter(np.float32(mid), np.float32(1e9))), "fp8") == grid[k + 1]
+            assert oracle.exchanged(float(np.nextafter(np.float32(mid), np.float32(0))), "fp8") == x
+    assert oracle.exchanged(460.0, "fp8") == 448.0 and oracle.exchanged(-1e9, "fp8") == -448.0
+    assert oracle.exchanged(2.0 ** -11, "fp8") == 0.0    # below half the smallest subnormal
+    rng = np.random.default_rng(6)
+    xs = (rng.standard_normal(20000) * np.exp(rng.standard_normal(20000) * 3)).astype(np.float32)
+    xs = xs[np.abs(xs) <= 448]
+    ref = torch.tensor(xs).to(torch.float8_e4m3fn).to(torch.float32).numpy()
+    got = np.array([oracle.exchanged(float(x), "fp8") for x in xs], dtype=np.float32)
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+
+
+@pytest.mark.parametrize("tau", [0, 2])
+def test_bruteforce_trace_with_fp8_exchange(tau):
+    R, N, T, seed = 3, 16, 8, 0x9A
+    w0, grads = rand_setup(R, N, T, seed=33)
+    o = oracle.Oracle(R, [N], p=0.5, tau=tau, ema_beta=0.6, seed=seed, lookahead_delay=[1],
+                      exchange="fp8", **HP)
+    ref = oracle.Oracle(R, [N], p=0.5, tau=tau, ema_beta=0.6, seed=seed, lookahead_delay=[1], **HP)
+    o.init_params(0, w0); ref.init_params(0, w0)
+    args = (R, N, 0.5, tau, 0.6, HP["lr"], HP["beta1"], HP["beta2"], HP["eps"],
+            HP["weight_decay"], seed, 1, w0, grads)
+    tr = bruteforce.run(np.float32, *args, wire="fp8")
+    for t in range(1, T + 1):
+        o.step([grads[t - 1]]); ref.step([grads[t - 1]])
+        for name in ("w", "m", "v", "d", "look"):
+            assert (o.get(0, name).astype(np.float64) == tr[t - 1][name]).all(), (t, name)
+    diff = np.abs(o.get(0, "w") - ref.get(0, "w")).max()
+    assert 1e-4 < diff < 1e-2     # about an E4M3 step (2^-4 relative) of |w| ~ 0.05
+
+
+# ---- eager staleness estimate (end of Section 3.2) --------------------------------
+
+@pytest.mark.parametrize("p,tau,K", [(1.0, 2, 2), (1.0, 3, 3), (0.5, 2, 1)])
+def test_eager_estimate_bruteforce_and_closed_form(p, tau, K):
+    R, N, T, seed = 3, 16, 10, 0x51
+    w0, grads = rand_setup(R, N, T, seed=41)
+    o = oracle.Oracle(R, [N], p=p, tau=tau, ema_beta=0.3, seed=seed, lookahead_delay=[1],
+                      avg_interval=K, correction="eager", **HP)
+    o.init_params(0, w0)
+    args = (R, N, p, tau, 0.3, HP["lr"], HP["beta1"], HP["beta2"], HP["eps"],
+            HP["weight_decay"], seed, 1, w0, grads)
+    tr = bruteforce.run(np.float32, *args, interval=K, correction="eager")
+    hist = {}
+    rounds = 0
+    for t in range(1, T + 1):
+        o.step([grads[t - 1]])
+        hist[t] = o.get(0, "what")
+        for name in ("w", "m", "v", "d", "look"):
+            assert (o.get(0, name).astype(np.float64) == tr[t - 1][name]).all(), (t, name)
+        if t % K == 0 and t > tau:
+            # closed form in double: w_i = mean_k w^_k^{t-tau} + (w^_i^t - w^_i^{t-tau}) / R
+            sel = o.subset_mask(0, t - tau)
+            old, now = hist[t - tau].astype(np.float64), hist[t].astype(np.float64)
+            want = old.mean(axis=0) + (now - old) / R
+            got = o.get(0, "w").astype(np.float64)
+            assert np.abs(got[:, sel] - want[:, sel]).max() < 3e-8
+            assert (got[:, ~sel] == now[:, ~sel]).all()
+            # the replica mean moves by 1/R of the mean progress made since t - tau
+            assert np.abs(got[:, sel].mean(axis=0)
+                          - (old.mean(axis=0) + (now.mean(axis=0) - old.mean(axis=0)) / R)[sel]).max() < 3e-8
+            rounds += 1
+    assert rounds > 0
+
+
+def test_eager_estimate_ignores_lambda_and_differs_from_the_ema():
+    R, N, T = 4, 64, 6
+    w0, grads = rand_setup(R, N, T, seed=43)
+    runs = {}
+    for name, kw in {"eager_a": dict(correction="eager", ema_beta=0.1),
+                     "eager_b": dict(correction="eager", ema_beta=0.9),
+                     "ema": dict(correction="ema", ema_beta=0.9)}.items():
+        o = oracle.Oracle(R, [N], p=1.0, tau=2, seed=3, avg_interval=2, **kw, **HP)
+        o.init_params(0, w0)
+        for t in range(T):
+            o.step([grads[t]])
+        runs[name] = o.get(0, "w")
+    assert (runs["eager_a"] == runs["eager_b"]).all()
+    assert (runs["eager_a"] != runs["ema"]).any()
+
+
+# ---- spread of the staleness estimates across replicas ------------------------------
+
+def test_ema_variance_against_numpy():
+    R, N, T = 4, 256, 9
+    w0, grads = rand_setup(R, N, T, seed=47)
+    o = oracle.Oracle(R, [N], p=0.5, tau=2, ema_beta=0.5, seed=11, **HP)
+    o.init_params(0, w0)
+    assert o.ema_variance(0) == (0.0, 0.0)
+    for t in range(T):
+        o.step([grads[t]])
+    var = o.get(0, "d").astype(np.float64).var(axis=0)      # population variance over replicas
+    mean, mx = o.ema_variance(0)
+    assert mx > 0 and abs(mean - var.mean()) <= 1e-12 * var.mean() and abs(mx - var.max()) <= 1e-12 * mx
+    # identical replicas (same gradients everywhere): the estimates agree, variance 0
+    o2 = oracle.Oracle(R, [N], p=0.5, tau=2, ema_beta=0.5, seed=11, **HP)
+    o2.init_params(0, w0)
+    for t in range(T):
+        o2.step([np.repeat(grads[t][:1], R, axis=0)])
+    assert np.abs(o2.get(0, "d")).max() > 0 and o2.ema_variance(0) == (0.0, 0.0)
+
+
 # ---- P9: elementwise independence ---------------------------------------------------
 
 def test_coordinate_slice_evolves_like_the_full_vector():
