@@ -49,6 +49,13 @@ extern "C" {
 #define ASYNCMESH_OPT_ADAMW 0u
 #define ASYNCMESH_OPT_NADAMW 1u
 
+/* asyncmesh_config.correction: the staleness estimate d_i of Section 3.2 */
+#define ASYNCMESH_CORRECTION_EMA 0u   /* Eq. "ema": d <- (1 - lambda) d + lambda (w^_i^t - w^_i^{t-tau}) */
+#define ASYNCMESH_CORRECTION_EAGER 1u /* d = (w^_i^t - w^_i^{t-tau}) / R, the eager-update rule the
+                                         section's last paragraph names as a special case (there with
+                                         p = 1 and tau = K; accepted here for any p, tau, K); lambda
+                                         is ignored                                                */
+
 /* asyncmesh_config.flags */
 #define ASYNCMESH_FLAG_SMALL_RING 1u /* diagnostic: give each compact ring slot 1/8 of
                                         its normal capacity, so that the overflow
@@ -62,6 +69,10 @@ extern "C" {
                                            replica average is first rounded to bfloat16 (nearest
                                            even); the average is formed in fp32 and a replica's own
                                            staleness sample uses its own unrounded value         */
+#define ASYNCMESH_FLAG_FP8_EXCHANGE 64u /* as BF16_EXCHANGE, with 8-bit floating point (E4M3: 4
+                                          exponent and 3 mantissa bits, nearest even, magnitudes above
+                                          448 clamp to 448, no scale factor; the paper does not say
+                                          which 8-bit format it used).  Not together with BF16_EXCHANGE */
 #define ASYNCMESH_FLAG_DENSE_RING 32u /* keep the snapshot ring dense (one position per coordinate
                                         and replica, tau slots) whatever p is: more memory and
                                         some more traffic, no compaction work                   */
@@ -110,7 +121,7 @@ typedef struct asyncmesh_config {
                                         Nesterov momentum and decoupled decay, the optimizer the
                                         paper runs asynchronous pipelines with (Appendix B.1,
                                         momentum beta1 = 0.99)                             */
-    uint32_t pad0;                   /* must be 0                                       */
+    uint32_t correction;             /* ASYNCMESH_CORRECTION_EMA (0) or ASYNCMESH_CORRECTION_EAGER */
     double momentum_decay;           /* NAdamW: psi of mu_t = beta1 (1 - 0.5 * 0.96^(t psi));
                                         0 selects the customary 0.004                   */
 } asyncmesh_config;
@@ -212,6 +223,16 @@ int asyncmesh_subset_mask(asyncmesh *h, uint32_t stage, uint64_t step,
  * the device in double precision.  Waits for the stream.
  */
 int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *out_host);
+
+/*
+ * Spread of the staleness estimates across replicas (the appendix figure on the
+ * consensus error plots the "variance between EMA estimates in each replica",
+ * mean and max across the model dimension): per coordinate the population
+ * variance (1/R) sum_i (d_i - dbar)^2, formed in double on the device;
+ * *mean_host = its mean over the stage's coordinates, *max_host = its maximum
+ * (host doubles, both required).  Waits for the stream.
+ */
+int asyncmesh_ema_variance(asyncmesh *h, uint32_t stage, double *mean_host, double *max_host);
 
 /*
  * The same quantity for callers that cannot let the library allocate (the paper

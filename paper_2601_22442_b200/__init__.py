@@ -9,6 +9,7 @@ from .binding import (AsyncMesh, AsyncMeshError, TorchAllocator, asyncmesh_creat
                       asyncmesh_read_params, asyncmesh_read_state, asyncmesh_read_state_range,
                       asyncmesh_subset_mask,
                       asyncmesh_consensus_error, asyncmesh_consensus_error_noalloc,
+                      asyncmesh_ema_variance,
                       asyncmesh_debug_philox,
                       asyncmesh_last_error, load)
 from .layouts import DEFAULT_HP, llama_stage_numel, workloads  # noqa: F401

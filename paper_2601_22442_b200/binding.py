@@ -23,6 +23,7 @@ FLAG_DIRECT_KERNEL = 2
 FLAG_PIPELINED_KERNEL = 4
 FLAG_BF16_EXCHANGE = 16
 FLAG_DENSE_RING = 32
+FLAG_FP8_EXCHANGE = 64
 STATE = {"w": 0, "m": 1, "v": 2, "d": 3, "look": 4}
 
 ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t)
@@ -44,7 +45,7 @@ class Config(ctypes.Structure):
         ("device", ctypes.c_int32), ("avg_interval", ctypes.c_int32),
         ("stream", ctypes.c_void_p),
         ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_ctx", ctypes.c_void_p),
-        ("optimizer", ctypes.c_uint32), ("pad0", ctypes.c_uint32),
+        ("optimizer", ctypes.c_uint32), ("correction", ctypes.c_uint32),
         ("momentum_decay", ctypes.c_double),
     ]
 
@@ -75,6 +76,8 @@ SIGNATURES = {
     "asyncmesh_read_state_range": (_int, [_vp, _u32, _int, _i32, _u64, _u64, _vp, _int]),
     "asyncmesh_subset_mask": (_int, [_vp, _u32, _u64, _vp]),
     "asyncmesh_consensus_error": (_int, [_vp, _u32, ctypes.POINTER(ctypes.c_double)]),
+    "asyncmesh_ema_variance": (_int, [_vp, _u32, ctypes.POINTER(ctypes.c_double),
+                                      ctypes.POINTER(ctypes.c_double)]),
     "asyncmesh_consensus_error_noalloc": (_int, [_int, _vp, _vp, _u32, _u64, _u64,
                                                  ctypes.POINTER(ctypes.c_double)]),
     "asyncmesh_step_count": (_int, [_vp, ctypes.POINTER(_u64)]),
@@ -154,7 +157,8 @@ class AsyncMesh:
                  device: int = 0, stream: Optional[int] = None,
                  allocator: Optional[TorchAllocator] = None,
                  use_torch_allocator: bool = True, flags: int = 0, avg_interval: int = 1,
-                 optimizer: str = "adamw", momentum_decay: float = 4e-3):
+                 optimizer: str = "adamw", momentum_decay: float = 4e-3,
+                 correction: str = "ema"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("asyncmesh needs a CUDA device; there is no CPU path")
@@ -182,7 +186,8 @@ class AsyncMesh:
             cfg.lookahead_delay = ctypes.cast(dl, ctypes.POINTER(ctypes.c_uint32))
         cfg.device, cfg.avg_interval, cfg.stream = self.device, int(avg_interval), stream
         cfg.optimizer = {"adamw": 0, "nadamw": 1}[optimizer]
-        cfg.pad0, cfg.momentum_decay = 0, float(momentum_decay)
+        cfg.correction = {"ema": 0, "eager": 1}[correction]
+        cfg.momentum_decay = float(momentum_decay)
         if self.allocator is not None:
             cfg.alloc, cfg.free = self.allocator.alloc_cb, self.allocator.free_cb
         h = _vp()
@@ -313,6 +318,12 @@ class AsyncMesh:
         _check(load().asyncmesh_consensus_error(self._h, stage, ctypes.byref(out)))
         return float(out.value)
 
+    def ema_variance(self, stage: int) -> tuple:
+        """(mean, max) over the stage's coordinates of the across-replica variance of d."""
+        mean, mx = ctypes.c_double(), ctypes.c_double()
+        _check(load().asyncmesh_ema_variance(self._h, stage, ctypes.byref(mean), ctypes.byref(mx)))
+        return float(mean.value), float(mx.value)
+
     @property
     def step_count(self) -> int:
         out = _u64()
@@ -374,6 +385,10 @@ def asyncmesh_read_state_range(h: AsyncMesh, stage, which, replica, first, count
 
 def asyncmesh_subset_mask(h: AsyncMesh, stage, step):
     return h.subset_mask(stage, step)
+
+
+def asyncmesh_ema_variance(h: AsyncMesh, stage):
+    return h.ema_variance(stage)
 
 
 def asyncmesh_consensus_error(h: AsyncMesh, stage):

@@ -14,7 +14,7 @@
 #include <cuda_runtime.h>
 
 #include "step_kernel.cuh"
-#include "step_kernel_pipelined.cuh"
+#include "kernel_table.cuh"
 
 using namespace amk;
 
@@ -65,19 +65,10 @@ struct DeviceScope {   // make the handle's device current for the call
 // the handle
 // ---------------------------------------------------------------------------
 
-typedef void (*step_fn)(const StepParams);
-
-
-struct KernelChoice {
-    step_fn fn = nullptr;
-    size_t smem = 0;              // dynamic shared memory per block
-    int threads = kBlockThreads;  // block size
-};
-
-
 struct asyncmesh {
     uint32_t R = 0, S = 0, tau = 0;
-    uint32_t wire_bf16 = 0;           // ASYNCMESH_FLAG_BF16_EXCHANGE
+    uint32_t wire = 0;                // 0 fp32, 1 ASYNCMESH_FLAG_BF16_EXCHANGE, 2 ASYNCMESH_FLAG_FP8_EXCHANGE
+    uint32_t correction = 0;          // ASYNCMESH_CORRECTION_*
     uint32_t optimizer = 0;           // ASYNCMESH_OPT_*
     double momentum_decay = 4e-3, mu_product = 1.0;   // NAdamW's momentum schedule
     uint32_t K = 1;                   // averaging interval in steps; tau is a multiple of it
@@ -210,6 +201,54 @@ __global__ void consensus_kernel(const float *W, uint32_t R, uint64_t stride, ui
     }
 }
 
+// Per coordinate the population variance of d over the replicas, in double;
+// out[0] accumulates the sum over coordinates, out[1] the maximum (variances are
+// non-negative, so their bit patterns order like unsigned integers).
+__global__ void spread_kernel(const float *D, uint32_t R, uint64_t coord_step, uint64_t replica_step,
+                              uint64_t N, double *out)
+{
+    double acc = 0.0, mx = 0.0;
+    for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
+         mu += (uint64_t)gridDim.x * blockDim.x) {
+        const float *p = D + mu * coord_step;
+        double mean = 0.0;
+        for (uint32_t i = 0; i < R; ++i) mean += (double)p[(uint64_t)i * replica_step];
+        mean /= (double)R;
+        double var = 0.0;
+        for (uint32_t i = 0; i < R; ++i) {
+            const double e = (double)p[(uint64_t)i * replica_step] - mean;
+            var += e * e;
+        }
+        var /= (double)R;
+        acc += var;
+        mx = var > mx ? var : mx;
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+        const double o = __shfl_down_sync(0xFFFFFFFFu, mx, d);
+        mx = o > mx ? o : mx;
+    }
+    __shared__ double part[32], pmax[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { part[warp] = acc; pmax[warp] = mx; }
+    __syncthreads();
+    if (warp == 0) {
+        const bool have = lane < (int)(blockDim.x >> 5);
+        acc = have ? part[lane] : 0.0;
+        mx = have ? pmax[lane] : 0.0;
+        for (int d = 16; d > 0; d >>= 1) {
+            acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+            const double o = __shfl_down_sync(0xFFFFFFFFu, mx, d);
+            mx = o > mx ? o : mx;
+        }
+        if (lane == 0) {
+            atomicAdd(out, acc);
+            atomicMax(reinterpret_cast<unsigned long long *>(out + 1),
+                      (unsigned long long)__double_as_longlong(mx));
+        }
+    }
+}
+
 __global__ void philox_debug_kernel(const uint32_t *ctr, const uint32_t *key, uint32_t *out,
                                     uint64_t n)
 {
@@ -233,61 +272,11 @@ static int grid_for(uint64_t items, int threads)
 // kernel dispatch
 // ---------------------------------------------------------------------------
 
-template <int R>
-static KernelChoice pick_mode(int mode, int pipelined, uint32_t S)
+static KernelChoice pick_kernel(uint32_t R, int mode, int pipelined, bool general, uint32_t S)
 {
-    KernelChoice c;
-    switch (mode) {
-    case kSync:
-        if (pipelined == 3) {
-            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeNarrow, kSync>;
-            c.threads = kPipeThreads;
-            c.smem = (size_t)pipe_table_bytes(S) +
-                     (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeNarrow>::warp_bytes(kPipeStages);
-        } else {
-            c.fn = asyncmesh_step_kernel<R, kSync>;
-        }
-        break;
-    case kDense: c.fn = asyncmesh_step_kernel<R, kDense>; break;
-    default:
-        if (pipelined == 1) {
-            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeWide, kCompact>;
-            c.threads = kPipeThreads;
-            c.smem = (size_t)pipe_table_bytes(S) +
-                     (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeWide>::warp_bytes(kPipeStages);
-        } else if (pipelined == 2) {
-            c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, PipeNarrow, kCompact>;
-            c.threads = kPipeThreads;
-            c.smem = (size_t)pipe_table_bytes(S) +
-                     (size_t)(kPipeThreads / 32) * PipeCfg<R, PipeNarrow>::warp_bytes(kPipeStages);
-        } else {
-            c.fn = asyncmesh_step_kernel<R, kCompact>;
-        }
-    }
-    return c;
-}
-
-static KernelChoice pick_kernel(uint32_t R, int mode, int pipelined, uint32_t S)
-{
-    switch (R) {
-    case 1: return pick_mode<1>(mode, pipelined, S);
-    case 2: return pick_mode<2>(mode, pipelined, S);
-    case 3: return pick_mode<3>(mode, pipelined, S);
-    case 4: return pick_mode<4>(mode, pipelined, S);
-    case 5: return pick_mode<5>(mode, pipelined, S);
-    case 6: return pick_mode<6>(mode, pipelined, S);
-    case 7: return pick_mode<7>(mode, pipelined, S);
-    case 8: return pick_mode<8>(mode, pipelined, S);
-    case 9: return pick_mode<9>(mode, pipelined, S);
-    case 10: return pick_mode<10>(mode, pipelined, S);
-    case 11: return pick_mode<11>(mode, pipelined, S);
-    case 12: return pick_mode<12>(mode, pipelined, S);
-    case 13: return pick_mode<13>(mode, pipelined, S);
-    case 14: return pick_mode<14>(mode, pipelined, S);
-    case 15: return pick_mode<15>(mode, pipelined, S);
-    case 16: return pick_mode<16>(mode, pipelined, S);
-    default: return KernelChoice();
-    }
+    if (pipelined) return R <= 8 ? pick_pipelined_few(R, pipelined, S) : pick_pipelined_many(R, pipelined, S);
+    if (R <= 8) return pick_direct_few(R, mode, general);
+    return general ? pick_direct_many_general(R, mode) : pick_direct_many_common(R, mode);
 }
 
 // The pipelined kernel stashes the selected coordinates of a sub-iteration
@@ -330,11 +319,15 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: betas must lie in [0, 1)");
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
                         ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE |
-                        ASYNCMESH_FLAG_DENSE_RING)) != 0)
+                        ASYNCMESH_FLAG_DENSE_RING | ASYNCMESH_FLAG_FP8_EXCHANGE)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
-    if (cfg->optimizer > ASYNCMESH_OPT_NADAMW || cfg->pad0 != 0 || !(cfg->momentum_decay >= 0.0))
+    if ((cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) && (cfg->flags & ASYNCMESH_FLAG_FP8_EXCHANGE))
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "create: BF16_EXCHANGE and FP8_EXCHANGE exclude each other");
+    if (cfg->optimizer > ASYNCMESH_OPT_NADAMW || cfg->correction > ASYNCMESH_CORRECTION_EAGER ||
+        !(cfg->momentum_decay >= 0.0))
         return fail(ASYNCMESH_ERR_INVALID_ARG,
-                    "create: optimizer must be 0 (AdamW) or 1 (NAdamW), pad0 0, momentum_decay >= 0");
+                    "create: optimizer must be 0 (AdamW) or 1 (NAdamW), correction 0 (EMA) or 1 (eager), "
+                    "momentum_decay >= 0");
     const uint32_t K = cfg->avg_interval < 1 ? 1u : (uint32_t)cfg->avg_interval;
     if (cfg->avg_interval < 0 || cfg->tau % K != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG,
@@ -362,7 +355,9 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     h->R = cfg->R; h->S = cfg->S; h->tau = cfg->tau;
     h->K = K; h->lag = cfg->tau / K;
     h->optimizer = cfg->optimizer;
-    h->wire_bf16 = (cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) ? 1u : 0u;
+    h->wire = (cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) ? 1u
+              : (cfg->flags & ASYNCMESH_FLAG_FP8_EXCHANGE) ? 2u : 0u;
+    h->correction = cfg->correction;
     h->momentum_decay = cfg->momentum_decay > 0.0 ? cfg->momentum_decay : 4e-3;
     h->p = cfg->p; h->ema_beta = cfg->ema_beta; h->lr = cfg->lr;
     h->beta1 = cfg->beta1; h->beta2 = cfg->beta2; h->eps = cfg->eps; h->wd = cfg->weight_decay;
@@ -434,6 +429,10 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
             h->pipelined = 2;
     }
 
+    // E4M3 exchange and the eager estimate exist in the direct kernel only
+    const bool general = h->wire == 2u || h->correction == ASYNCMESH_CORRECTION_EAGER;
+    if (general) h->pipelined = 0;
+
     auto bail = [&](int code, const char *what) {
         release_all(h);
         delete h;
@@ -497,7 +496,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
 
     // persistent grid: every SM filled to the kernel's occupancy
-    h->kernel = pick_kernel(R, h->mode, h->pipelined, S);
+    h->kernel = pick_kernel(R, h->mode, h->pipelined, general, S);
     int sms = 0, per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
     cudaError_t ke = cudaSuccess;
@@ -621,7 +620,8 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.lam = (float)lam;
     P.oml = (float)(1.0 - lam);
     P.Rf = (float)h->R;
-    P.wire_bf16 = h->wire_bf16;
+    P.wire = h->wire;
+    P.eager = h->correction == ASYNCMESH_CORRECTION_EAGER ? 1u : 0u;
     P.nesterov = h->optimizer == ASYNCMESH_OPT_NADAMW ? 1u : 0u;
     double mu_product = h->mu_product;
     if (P.nesterov) {   // mu_t, mu_{t+1} and the running product of the momentum schedule
@@ -840,6 +840,28 @@ extern "C" int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *o
     CU_TRY(cudaGetLastError());
     CU_TRY(cudaMemcpyAsync(out_host, h->scratch, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
     CU_TRY(cudaStreamSynchronize(h->stream));
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_ema_variance(asyncmesh *h, uint32_t stage, double *mean_host,
+                                      double *max_host)
+{
+    if (!h || !mean_host || !max_host || stage >= h->S)
+        return fail(ASYNCMESH_ERR_INVALID_ARG, "ema_variance: bad handle, stage or output");
+    DeviceScope scope(h->device);
+    const StageDesc &d = h->sd[stage];
+    // d is coordinate-major [stride][R] except with the dense ring ([R][stride])
+    const uint64_t coord_step = h->mode == kDense ? 1 : h->R;
+    const uint64_t replica_step = h->mode == kDense ? d.stride : 1;
+    CU_TRY(cudaMemsetAsync(h->scratch, 0, 2 * sizeof(double), h->stream));
+    spread_kernel<<<grid_for(d.N, 256), 256, 0, h->stream>>>(d.D, h->R, coord_step, replica_step, d.N,
+                                                             h->scratch);
+    CU_TRY(cudaGetLastError());
+    double out[2];
+    CU_TRY(cudaMemcpyAsync(out, h->scratch, sizeof out, cudaMemcpyDeviceToHost, h->stream));
+    CU_TRY(cudaStreamSynchronize(h->stream));
+    *mean_host = out[0] / (double)d.N;
+    *max_host = out[1];
     return ASYNCMESH_OK;
 }
 

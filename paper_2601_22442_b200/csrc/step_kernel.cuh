@@ -33,6 +33,8 @@
 #pragma once
 #include <cstdint>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
 #include "philox.cuh"
@@ -78,7 +80,9 @@ struct StepParams {
     uint32_t prod_slot, cons_slot;
     SubsetRule rule;
     float b1, b2, omb1, omb2, ib1, ib2, eps, lr, lrwd, lam, oml, Rf;
-    uint32_t wire_bf16;          // snapshots enter the average rounded to bfloat16
+    uint32_t wire;               // snapshots enter the average as fp32 (0), rounded to bfloat16 (1)
+                                 // or to 8-bit floating point E4M3 (2)
+    uint32_t eager;              // staleness estimate: 0 Eq. "ema", 1 d = (w^ - w^_old) / R
     uint32_t nesterov;           // 0: AdamW, 1: NAdamW
     float cg, cm;                // NAdamW: weights of the gradient and momentum parts
 };
@@ -93,12 +97,35 @@ __device__ __forceinline__ void st_stream(float *p, const float (&x)[4])
 }
 
 // A snapshot value as the other replicas see it: unchanged, or rounded to
-// bfloat16 (round to nearest even) when the subset is exchanged in reduced
-// precision (the paper's quantisation study).  The average is formed in fp32; a
-// replica's own staleness sample keeps using its own unrounded value.
+// bfloat16 or to E4M3 (round to nearest even; E4M3 clamps at its largest finite
+// value 448) when the subset is exchanged in reduced precision (the paper's
+// quantisation study).  The average is formed in fp32; a replica's own
+// staleness sample keeps using its own unrounded value.
+// GEN selects the general form (also E4M3, also the eager estimate below); the
+// kernels of the common configurations are compiled without it: the pipelined
+// kernel's run time moves by several percent with a handful of extra instructions
+// in its sparse phase (measured: +7 % inline, +2 % as out-of-line calls).
+template <bool GEN>
 __device__ __forceinline__ float on_wire(const StepParams &P, float x)
 {
-    return P.wire_bf16 ? __bfloat162float(__float2bfloat16_rn(x)) : x;
+    if constexpr (GEN) {
+        if (P.wire == 2u) {
+            const __nv_fp8_storage_t q = __nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3);
+            return __half2float(__half(__nv_cvt_fp8_to_halfraw(q, __NV_E4M3)));
+        }
+    }
+    return P.wire ? __bfloat162float(__float2bfloat16_rn(x)) : x;
+}
+
+// The staleness estimate of a consumed coordinate (Section 3.2): Eq. "ema", or the
+// eager estimate the section's last paragraph names as a special case.
+template <bool GEN>
+__device__ __forceinline__ float staleness(const StepParams &P, float d, float diff)
+{
+    if constexpr (GEN) {
+        if (P.eager) return __fdiv_rn(diff, P.Rf);
+    }
+    return __fadd_rn(__fmul_rn(P.oml, d), __fmul_rn(P.lam, diff));
 }
 
 // The local optimizer step (first line of Eq. "sparta"), one rounding per written
@@ -157,7 +184,7 @@ __device__ __forceinline__ uint32_t warp_exclusive_sum(uint32_t x, int lane, uin
     return incl - x;
 }
 
-template <int R, int MODE>
+template <int R, int MODE, bool GEN>
 __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDesc &st,
                                               const float *__restrict__ G, uint32_t s,
                                               uint32_t chunk, int lane)
@@ -258,7 +285,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                         const float r[4] = {r4[i].x, r4[i].y, r4[i].z, r4[i].w};
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
-                            a[c] = (i == 0) ? on_wire(P, r[c]) : __fadd_rn(a[c], on_wire(P, r[c]));
+                            a[c] = (i == 0) ? on_wire<GEN>(P, r[c]) : __fadd_rn(a[c], on_wire<GEN>(P, r[c]));
                     }
 #pragma unroll
                     for (int c = 0; c < 4; ++c) abar[c] = __fdiv_rn(a[c], P.Rf);
@@ -286,7 +313,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                         for (int c = 0; c < 4; ++c) {
                             if ((cm >> c) & 1u) {
                                 const float diff = __fsub_rn(wh[c], old[c]);
-                                dd[c] = __fadd_rn(__fmul_rn(P.oml, dd[c]), __fmul_rn(P.lam, diff));
+                                dd[c] = staleness<GEN>(P, dd[c], diff);
                                 wn[c] = __fadd_rn(abar[c], dd[c]);
                             }
                         }
@@ -321,9 +348,9 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                         ce[j] = idx * R;
                         float old[R];
                         load_replicas<R>(ring_cons + ce[j], old);
-                        float a = on_wire(P, old[0]);
+                        float a = on_wire<GEN>(P, old[0]);
 #pragma unroll
-                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire(P, old[i]));
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire<GEN>(P, old[i]));
                         abar[j] = __fdiv_rn(a, P.Rf);
                     }
                 }
@@ -394,8 +421,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                         for (int j = 0; j < 4; ++j) {
                             if ((cm >> j) & 1u) {
                                 const float diff = __fsub_rn(wh[j], old[ii][j]);
-                                const float dn = __fadd_rn(__fmul_rn(P.oml, dd[ii][j]),
-                                                           __fmul_rn(P.lam, diff));
+                                const float dn = staleness<GEN>(P, dd[ii][j], diff);
                                 st.D[(mu + j) * R + i] = dn;
                                 wn[j] = __fadd_rn(abar[j], dn);
                             }
@@ -410,7 +436,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                 } else {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        acc[c] = (i == 0) ? on_wire(P, wh[c]) : __fadd_rn(acc[c], on_wire(P, wh[c]));
+                        acc[c] = (i == 0) ? on_wire<GEN>(P, wh[c]) : __fadd_rn(acc[c], on_wire<GEN>(P, wh[c]));
                         wold_keep[i][c] = w[c];
                     }
                 }
@@ -471,7 +497,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
     }
 }
 
-template <int R, int MODE>
+template <int R, int MODE, bool GEN>
 __global__ void __launch_bounds__(kBlockThreads)
 asyncmesh_step_kernel(const __grid_constant__ StepParams P)
 {
@@ -491,7 +517,7 @@ asyncmesh_step_kernel(const __grid_constant__ StepParams P)
     for (uint32_t gc = blockIdx.x * wpb + (threadIdx.x >> 5); gc < P.total_chunks;
          gc += n_warps) {
         while (s + 1 < P.S && gc >= sd[s + 1].chunk_begin) ++s;
-        process_chunk<R, MODE>(P, sd[s], P.G[s], s, gc - sd[s].chunk_begin, lane);
+        process_chunk<R, MODE, GEN>(P, sd[s], P.G[s], s, gc - sd[s].chunk_begin, lane);
     }
 }
 

@@ -1,0 +1,126 @@
+// Instantiations of the step kernels.  Compiled five times, -DAM_PART=0..4:
+// 0 direct kernel R = 1..8; 1 direct kernel R = 9..16, common form; 2 the same,
+// general form; 3 pipelined kernel R = 1..8; 4 pipelined kernel R = 9..16.
+#include "kernel_table.cuh"
+
+#ifndef AM_PART
+#error "compile with -DAM_PART=0..4"
+#endif
+
+namespace amk {
+
+#if AM_PART < 3
+
+template <int R, bool GEN>
+static KernelChoice direct_as(int mode)
+{
+    KernelChoice c;
+    switch (mode) {
+    case kSync: c.fn = asyncmesh_step_kernel<R, kSync, GEN>; break;
+    case kDense: c.fn = asyncmesh_step_kernel<R, kDense, GEN>; break;
+    default: c.fn = asyncmesh_step_kernel<R, kCompact, GEN>;
+    }
+    return c;
+}
+
+#if AM_PART == 0
+template <int R>
+static KernelChoice direct(int mode, bool general)
+{
+    return general ? direct_as<R, true>(mode) : direct_as<R, false>(mode);
+}
+KernelChoice pick_direct_few(uint32_t R, int mode, bool general)
+{
+    switch (R) {
+    case 1: return direct<1>(mode, general);
+    case 2: return direct<2>(mode, general);
+    case 3: return direct<3>(mode, general);
+    case 4: return direct<4>(mode, general);
+    case 5: return direct<5>(mode, general);
+    case 6: return direct<6>(mode, general);
+    case 7: return direct<7>(mode, general);
+    case 8: return direct<8>(mode, general);
+    default: return KernelChoice();
+    }
+}
+#else
+constexpr bool kGeneral = (AM_PART == 2);
+#if AM_PART == 1
+KernelChoice pick_direct_many_common(uint32_t R, int mode)
+#else
+KernelChoice pick_direct_many_general(uint32_t R, int mode)
+#endif
+{
+    switch (R) {
+    case 9: return direct_as<9, kGeneral>(mode);
+    case 10: return direct_as<10, kGeneral>(mode);
+    case 11: return direct_as<11, kGeneral>(mode);
+    case 12: return direct_as<12, kGeneral>(mode);
+    case 13: return direct_as<13, kGeneral>(mode);
+    case 14: return direct_as<14, kGeneral>(mode);
+    case 15: return direct_as<15, kGeneral>(mode);
+    case 16: return direct_as<16, kGeneral>(mode);
+    default: return KernelChoice();
+    }
+}
+#endif
+
+#else   // pipelined kernel
+
+template <int R, class SH, int MODE>
+static KernelChoice pipelined_as(uint32_t S)
+{
+    KernelChoice c;
+    c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, SH, MODE>;
+    c.threads = kPipeThreads;
+    c.smem = (size_t)pipe_table_bytes(S) +
+             (size_t)(kPipeThreads / 32) * PipeCfg<R, SH>::warp_bytes(kPipeStages);
+    return c;
+}
+
+template <int R>
+static KernelChoice pipelined(int shape, uint32_t S)
+{
+    switch (shape) {
+    case 1: return pipelined_as<R, PipeWide, kCompact>(S);
+    case 2: return pipelined_as<R, PipeNarrow, kCompact>(S);
+    case 3: return pipelined_as<R, PipeNarrow, kSync>(S);
+    default: return KernelChoice();
+    }
+}
+
+#if AM_PART == 3
+KernelChoice pick_pipelined_few(uint32_t R, int shape, uint32_t S)
+{
+    switch (R) {
+    case 1: return pipelined<1>(shape, S);
+    case 2: return pipelined<2>(shape, S);
+    case 3: return pipelined<3>(shape, S);
+    case 4: return pipelined<4>(shape, S);
+    case 5: return pipelined<5>(shape, S);
+    case 6: return pipelined<6>(shape, S);
+    case 7: return pipelined<7>(shape, S);
+    case 8: return pipelined<8>(shape, S);
+    default: return KernelChoice();
+    }
+}
+#else
+KernelChoice pick_pipelined_many(uint32_t R, int shape, uint32_t S)
+{
+    switch (R) {
+    case 9: return pipelined<9>(shape, S);
+    case 10: return pipelined<10>(shape, S);
+    case 11: return pipelined<11>(shape, S);
+    case 12: return pipelined<12>(shape, S);
+    case 13: return pipelined<13>(shape, S);
+    case 14: return pipelined<14>(shape, S);
+    case 15: return pipelined<15>(shape, S);
+    case 16: return pipelined<16>(shape, S);
+    default: return KernelChoice();
+    }
+}
+#endif
+
+#endif
+
+}  // namespace amk

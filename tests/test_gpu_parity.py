@@ -26,15 +26,15 @@ def am():
 
 
 def make_pair(R, numel, p, tau, lam, delays=None, seed=0x5EED, hp=HP, same_init=True,
-              init_seed=0x1217, flags=0, avg_interval=1, optimizer="adamw", exchange="fp32"):
-    if exchange == "bf16":
-        flags |= 16
+              init_seed=0x1217, flags=0, avg_interval=1, optimizer="adamw", exchange="fp32",
+              correction="ema"):
+    flags |= {"fp32": 0, "bf16": 16, "fp8": 64}[exchange]
     o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
                       lookahead_delay=delays, avg_interval=avg_interval, optimizer=optimizer,
-                      exchange=exchange, **hp)
+                      exchange=exchange, correction=correction, **hp)
     g = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
                        lookahead_delay=delays, flags=flags, avg_interval=avg_interval,
-                       optimizer=optimizer, **hp)
+                       optimizer=optimizer, correction=correction, **hp)
     for s, n in enumerate(numel):
         if same_init:
             w0 = si.init_weights_host(init_seed, s, 0, n)
@@ -210,6 +210,83 @@ def test_bf16_exchange(tau, p):
     for t in range(1, 3 * tau + 6):
         ref.step([si.grads_host(0x6AD5, t, s, 4, 0, n) for s, n in enumerate([6000, 1024 + 9])])
     assert np.abs(ref.get(0, "w") - g.get(0, "w")).max() > 0
+
+
+@pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (3, 0.4)])
+def test_fp8_exchange(tau, p):
+    # subsets exchanged in 8-bit floating point (E4M3): all ring modes, both compact-ring kernels
+    from paper_2601_22442_b200 import binding
+    o, g = run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 5, exchange="fp8")
+    run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="fp8",
+             flags=binding.FLAG_DIRECT_KERNEL)
+    ref = oracle.Oracle(4, [6000, 1024 + 9], p=p, tau=tau, ema_beta=0.9, exchange="bf16", **HP)
+    for s, n in enumerate([6000, 1024 + 9]):
+        ref.init_params(s, si.init_weights_host(0x1217, s, 0, n))
+    for t in range(1, 3 * tau + 6):
+        ref.step([si.grads_host(0x6AD5, t, s, 4, 0, n) for s, n in enumerate([6000, 1024 + 9])])
+    assert np.abs(ref.get(0, "w") - g.get(0, "w")).max() > 0    # nor is it the bfloat16 exchange
+
+
+def test_fp8_conversion_on_the_device_covers_the_whole_format():
+    # every E4M3 value, every midpoint between neighbours and its two fp32 neighbours pass
+    # through one synchronous averaging step with R = 1 and p = 1: the result is the
+    # snapshot as "the others" see it, i.e. the rounded value itself (mean of one, + 0)
+    grid = []
+    for e in range(16):
+        for mant in range(8):
+            if not (e == 15 and mant == 7):
+                grid.append(mant / 8 * 2.0 ** -6 if e == 0 else (1 + mant / 8) * 2.0 ** (e - 7))
+    xs = []
+    for k, x in enumerate(grid):
+        xs.append(x)
+        if k + 1 < len(grid):
+            mid = np.float32((x + grid[k + 1]) / 2)
+            xs += [float(mid), float(np.nextafter(mid, np.float32(1e9))), float(np.nextafter(mid, np.float32(0)))]
+    xs += [460.0, 1e6, 2.0 ** -11, 3e-5]
+    xs = np.array(xs + [-v for v in xs], dtype=np.float32)
+    hp = dict(HP, lr=1e-30, weight_decay=0.0)      # the optimizer step leaves w unchanged
+    o = oracle.Oracle(1, [xs.size], p=1.0, tau=0, ema_beta=0.9, exchange="fp8", **hp)
+    g = am().AsyncMesh(1, [xs.size], p=1.0, tau=0, ema_beta=0.9, flags=64, **hp)
+    o.init_params(0, xs); g.init_params(0, xs)
+    zero = np.zeros((1, xs.size), dtype=np.float32)
+    bufs = g.empty_grads()
+    bufs[0].zero_()
+    o.step([zero]); g.step(bufs)
+    want = np.array([oracle.exchanged(float(x), "fp8") for x in xs], dtype=np.float32)
+    assert np.array_equal(o.get(0, "w")[0], want)
+    assert np.array_equal(g.get(0, "w")[0], want)
+
+
+@pytest.mark.parametrize("p,tau,K", [(1.0, 2, 2), (1.0, 4, 4), (0.05, 2, 1), (0.3, 3, 3), (0.5, 0, 1)])
+def test_eager_staleness_estimate(p, tau, K):
+    # d = (w^_i^t - w^_i^{t-tau}) / R instead of Eq. "ema": dense ring (p = 1), both
+    # compact-ring kernels, synchronous mode (where the estimate is exactly 0 either way)
+    from paper_2601_22442_b200 import binding
+    steps = 3 * max(tau, K) + 4
+    o, g = run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=steps, avg_interval=K, correction="eager")
+    if tau:
+        assert np.abs(g.get(0, "d")).max() > 0
+    run_case(3, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
+             flags=binding.FLAG_DIRECT_KERNEL)
+    if 0 < p < 1 and tau:
+        run_case(3, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
+                 flags=binding.FLAG_DENSE_RING)
+
+
+@pytest.mark.parametrize("p,tau,flags", [(0.05, 2, 0), (0.3, 1, 0), (1.0, 2, 0), (0.3, 2, 2), (0.3, 0, 0)])
+def test_ema_variance_diagnostic(p, tau, flags):
+    o, g = run_case(4, [6000, 1024 + 9], p, tau, 0.5, steps=3 * tau + 6, flags=flags)
+    for s in range(2):
+        mean_o, max_o = o.ema_variance(s)
+        mean_g, max_g = g.ema_variance(s)
+        assert max_g == max_o                       # same double operations per coordinate
+        assert abs(mean_g - mean_o) <= 1e-12 * max(mean_o, 1e-300)
+        if tau:
+            assert max_o > 0
+        else:
+            assert (mean_o, max_o) == (0.0, 0.0)
+    again = am().asyncmesh_ema_variance(g, 1)     # (the sum's order is not fixed: last bits may move)
+    assert again[1] == max_g and abs(again[0] - mean_g) <= 1e-12 * max(mean_g, 1e-300)
 
 
 @pytest.mark.parametrize("lam", [0.0, 1.0])
