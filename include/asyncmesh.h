@@ -73,6 +73,10 @@ extern "C" {
                                           exponent and 3 mantissa bits, nearest even, magnitudes above
                                           448 clamp to 448, no scale factor; the paper does not say
                                           which 8-bit format it used).  Not together with BF16_EXCHANGE */
+#define ASYNCMESH_FLAG_KEEP_PREVIOUS 128u /* keep w^{t-1}: before each step the weights are copied
+                                            aside (one device-to-device copy per stage, 8 bytes per
+                                            replica-coordinate of extra traffic, 4 bytes of memory),
+                                            and asyncmesh_lookahead_weights accepts any delay    */
 #define ASYNCMESH_FLAG_DENSE_RING 32u /* keep the snapshot ring dense (one position per coordinate
                                         and replica, tau slots) whatever p is: more memory and
                                         some more traffic, no compaction work                   */
@@ -183,8 +187,12 @@ int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host);
 /*
  * Look-ahead weights of a stage: w^t + delay * (w^t - w^{t-1}) (Section 2.2).
  * Returns a library-owned device pointer [R][row_stride], valid until the next
- * step or destroy.  delay must be the stage's configured delay (the buffer the
- * fused step wrote) or 0 (the weights themselves); anything else: UNSUPPORTED.
+ * step, the next call for the same stage with another delay, or destroy.
+ * delay = the stage's configured delay: the buffer the fused step wrote; delay
+ * = 0: the weights themselves; any other delay: computed now, on the stream,
+ * into a per-stage buffer allocated on first use, from the weights and their
+ * previous values -- only if the handle was created with
+ * ASYNCMESH_FLAG_KEEP_PREVIOUS, otherwise UNSUPPORTED.
  */
 int asyncmesh_lookahead_weights(asyncmesh *h, uint32_t stage, uint32_t delay,
                                 const float **out_device, uint64_t *row_stride);

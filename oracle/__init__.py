@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.am_oracle_step_ex.argtypes = [vp, vp, dbl, dbl]
         L.am_oracle_row.restype = ctypes.POINTER(ctypes.c_float)
         L.am_oracle_row.argtypes = [vp, u32, ctypes.c_int, u32]
+        L.am_oracle_lookahead.restype = ctypes.c_int
+        L.am_oracle_lookahead.argtypes = [vp, u32, u32, vp]
         L.am_oracle_mean_params.restype = ctypes.c_int
         L.am_oracle_mean_params.argtypes = [vp, u32, vp]
         L.am_oracle_consensus_error.restype = dbl
@@ -191,6 +193,13 @@ class Oracle:
     def get(self, stage: int, which: str) -> np.ndarray:
         """All replicas of one state array: shape (R, numel[stage])."""
         return np.stack([self.row(stage, which, i) for i in range(self.R)])
+
+    def lookahead(self, stage: int, delay: int) -> np.ndarray:
+        """Look-ahead weights for any delay, shape (R, numel[stage])."""
+        out = np.empty((self.R, self.numel[stage]), dtype=np.float32)
+        if lib().am_oracle_lookahead(self._h, stage, int(delay), out.ctypes.data) != 0:
+            raise ValueError("oracle: bad lookahead request")
+        return out
 
     def mean_params(self, stage: int) -> np.ndarray:
         out = np.empty(self.numel[stage], dtype=np.float32)

@@ -422,6 +422,21 @@ const float *am_oracle_row(const am_oracle *o, uint32_t stage, int which,
     return a[stage] + (uint64_t)replica * o->numel[stage];
 }
 
+/* Look-ahead weights of a stage for any delay (Section 2.2): the same
+ * extrapolation as O4, w + delay (w - w^{t-1}), from the current and the
+ * previous weights.  dst receives [R][numel] floats. */
+int am_oracle_lookahead(const am_oracle *o, uint32_t stage, uint32_t delay, float *dst)
+{
+    if (!o || stage >= o->S || !dst) return -1;
+    const uint64_t n = (uint64_t)o->R * o->numel[stage];
+    const float delta = (float)delay;
+    for (uint64_t k = 0; k < n; ++k) {
+        const float dir = o->w[stage][k] - o->wprev[stage][k];
+        dst[k] = o->w[stage][k] + (delta * dir);
+    }
+    return 0;
+}
+
 /* Replica mean of the weights (the consensus model the paper evaluates):
  * sequential sum over i = 0..R-1, one division by (float) R. */
 int am_oracle_mean_params(const am_oracle *o, uint32_t stage, float *dst)

@@ -85,6 +85,8 @@ struct asyncmesh {
     std::vector<uint32_t> delay;
     std::vector<StageDesc> sd;        // host copy of the stage table
     std::vector<float *> gstage;      // staging gradients for asyncmesh_step_host
+    std::vector<float *> wprev;       // w^{t-1} per stage (ASYNCMESH_FLAG_KEEP_PREVIOUS)
+    std::vector<float *> lookx;       // look-ahead at a delay asked for after the fact, per stage
     std::vector<void *> owned;        // everything obtained from the allocator
 
     StageDesc *sd_dev = nullptr;
@@ -198,6 +200,23 @@ __global__ void consensus_kernel(const float *W, uint32_t R, uint64_t stride, ui
         acc = lane < (int)(blockDim.x >> 5) ? part[lane] : 0.0;
         for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
         if (lane == 0) atomicAdd(out, acc);
+    }
+}
+
+// look = w + delay (w - w_prev) (Section 2.2), float4 at a time (rows are padded to 32 floats).
+__global__ void extrapolate_kernel(const float *W, const float *Wprev, float *out, float delay,
+                                   uint64_t n4)
+{
+    for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n4;
+         k += (uint64_t)gridDim.x * blockDim.x) {
+        const float4 w = reinterpret_cast<const float4 *>(W)[k];
+        const float4 q = reinterpret_cast<const float4 *>(Wprev)[k];
+        float4 o;
+        o.x = __fadd_rn(w.x, __fmul_rn(delay, __fsub_rn(w.x, q.x)));
+        o.y = __fadd_rn(w.y, __fmul_rn(delay, __fsub_rn(w.y, q.y)));
+        o.z = __fadd_rn(w.z, __fmul_rn(delay, __fsub_rn(w.z, q.z)));
+        o.w = __fadd_rn(w.w, __fmul_rn(delay, __fsub_rn(w.w, q.w)));
+        reinterpret_cast<float4 *>(out)[k] = o;
     }
 }
 
@@ -319,7 +338,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: betas must lie in [0, 1)");
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
                         ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE |
-                        ASYNCMESH_FLAG_DENSE_RING | ASYNCMESH_FLAG_FP8_EXCHANGE)) != 0)
+                        ASYNCMESH_FLAG_DENSE_RING | ASYNCMESH_FLAG_FP8_EXCHANGE |
+                        ASYNCMESH_FLAG_KEEP_PREVIOUS)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
     if ((cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) && (cfg->flags & ASYNCMESH_FLAG_FP8_EXCHANGE))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: BF16_EXCHANGE and FP8_EXCHANGE exclude each other");
@@ -370,6 +390,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     h->delay.resize(S);
     h->sd.assign(S, StageDesc{});
     h->gstage.assign(S, nullptr);
+    h->wprev.assign(S, nullptr);
+    h->lookx.assign(S, nullptr);
 
     // subset rule: floor(p * 2^32) in double
     const double tf = std::floor(cfg->p * 4294967296.0);
@@ -459,6 +481,10 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         d.V = (float *)zalloc(row_bytes);
         d.D = (float *)zalloc(row_bytes);
         if (!d.W || !d.M || !d.V || !d.D) return bail(ASYNCMESH_ERR_OOM, "out of device memory (state)");
+        if (cfg->flags & ASYNCMESH_FLAG_KEEP_PREVIOUS) {
+            h->wprev[s] = (float *)zalloc(row_bytes);
+            if (!h->wprev[s]) return bail(ASYNCMESH_ERR_OOM, "out of device memory (previous weights)");
+        }
         d.LOOK = d.W;
         if (d.has_look) {
             d.LOOK = (float *)zalloc(row_bytes);
@@ -632,6 +658,11 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
         P.cm = (float)(lr * mu_n / (1.0 - mu_product * mu_n));
     }
 
+    for (uint32_t s = 0; s < h->S; ++s)   // w^{t-1} for look-aheads asked for after the fact
+        if (h->wprev[s])
+            CU_TRY(cudaMemcpyAsync(h->wprev[s], h->sd[s].W, (size_t)h->R * h->stride[s] * sizeof(float),
+                                   cudaMemcpyDeviceToDevice, h->stream));
+
     if (h->mode == kCompact && round)   // the producing slot's cursors start this step at zero
         CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
                                h->S * sizeof(unsigned int), h->stream));
@@ -713,12 +744,23 @@ extern "C" int asyncmesh_lookahead_weights(asyncmesh *h, uint32_t stage, uint32_
     if (!h || !out_device || !row_stride || stage >= h->S)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "lookahead_weights: bad handle, stage or output");
     const StageDesc &d = h->sd[stage];
-    if (delay == 0) *out_device = d.W;
+    if (delay == 0 || h->t == 0) *out_device = d.W;   // before the first step w^{-1} = w^0
     else if (delay == h->delay[stage]) *out_device = d.LOOK;
-    else
+    else if (h->wprev[stage]) {
+        DeviceScope scope(h->device);
+        const uint64_t n = (uint64_t)h->R * d.stride;
+        if (!h->lookx[stage]) {
+            h->lookx[stage] = (float *)dev_alloc(h, n * sizeof(float));
+            if (!h->lookx[stage]) return fail(ASYNCMESH_ERR_OOM, "lookahead_weights: out of device memory");
+        }
+        extrapolate_kernel<<<grid_for(n / 4, 256), 256, 0, h->stream>>>(d.W, h->wprev[stage], h->lookx[stage],
+                                                                       (float)delay, n / 4);
+        CU_TRY(cudaGetLastError());
+        *out_device = h->lookx[stage];
+    } else
         return fail(ASYNCMESH_ERR_UNSUPPORTED,
-                    "lookahead_weights: stage %u was configured with delay %u, not %u", stage,
-                    h->delay[stage], delay);
+                    "lookahead_weights: stage %u was configured with delay %u, not %u (any delay "
+                    "needs ASYNCMESH_FLAG_KEEP_PREVIOUS)", stage, h->delay[stage], delay);
     *row_stride = d.stride;
     return ASYNCMESH_OK;
 }

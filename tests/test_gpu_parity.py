@@ -332,6 +332,26 @@ def test_lookahead_pointers_and_default_delays():
     assert e.value.code == -5
 
 
+@pytest.mark.parametrize("p,tau", [(0.2, 2), (0.3, 0), (1.0, 1)])
+def test_lookahead_for_any_delay_with_kept_previous_weights(p, tau):
+    # ASYNCMESH_FLAG_KEEP_PREVIOUS: w^{t-1} is kept, any delay can be asked for afterwards
+    from paper_2601_22442_b200 import binding
+    numel = [1500, 1024 + 9]
+    o, g = make_pair(3, numel, p, tau, 0.9, delays=[2, 0], flags=binding.FLAG_KEEP_PREVIOUS)
+    ptr, stride = g.lookahead_weights(0, 5)          # before any step: the weights themselves
+    assert ptr == g.lookahead_weights(0, 0)[0]
+    bufs = None
+    for t in range(1, 2 * tau + 5):
+        bufs = step_both(o, g, t, bufs=bufs)
+        for s, n in enumerate(numel):
+            for delay in (1, 2, 7, 0):
+                ptr, stride = g.lookahead_weights(s, delay)
+                view = torch.as_tensor(DevicePtr(ptr, 3, stride), device="cuda")
+                assert np.array_equal(view[:, :n].cpu().numpy(), o.lookahead(s, delay)), (t, s, delay)
+    compare(o, g)                                    # and the step itself is unchanged by the copies
+    assert g.lookahead_weights(0, 2)[0] != g.lookahead_weights(0, 7)[0]   # configured delay: the fused buffer
+
+
 def test_step_host_equals_step():
     numel = [3000, 1025]
     a = am().AsyncMesh(3, numel, p=0.2, tau=1, ema_beta=0.9, **HP)

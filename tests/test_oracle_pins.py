@@ -331,6 +331,38 @@ def test_lookahead_default_delay_and_constant_velocity():
     assert (o.row(s, "look", 0) == (w + np.float32(2) * (w - wp)).astype(np.float32)).all()
 
 
+def test_lookahead_for_any_delay():
+    # delay 0 is the weights, the configured delay is what the step wrote, and under a
+    # constant update direction delay k lands on the weights k steps later
+    N, T = 129, 14
+    g = np.linspace(-1.0, 1.0, N).astype(np.float32)
+    g[np.abs(g) < 1e-3] = 0.25
+    o = oracle.Oracle(1, [N], p=0.0, tau=0, ema_beta=0.9, lookahead_delay=[3],
+                      **dict(HP, weight_decay=0.0))
+    o.init_params(0, np.zeros(N, dtype=np.float32))
+    assert (o.lookahead(0, 7) == o.get(0, "w")).all()        # before any step: w^{-1} = w^0
+    snap, ws = {}, {}
+    for t in range(1, T + 1):
+        o.step([g[None, :]])
+        ws[t] = o.get(0, "w")
+        assert (o.lookahead(0, 0) == ws[t]).all()
+        assert (o.lookahead(0, 3) == o.get(0, "look")).all()
+        if t == 5:
+            snap = {k: o.lookahead(0, k) for k in (1, 2, 6, 9)}
+    for k, look in snap.items():
+        assert np.abs(look - ws[5 + k]).max() < 1e-6 * np.abs(ws[5 + k]).max()
+    # a brute-force trace agrees with the oracle's own look at a delay both computed
+    R, N2, seed = 2, 16, 0xABC
+    w0, grads = rand_setup(R, N2, 4, seed=9)
+    o2 = oracle.Oracle(R, [N2], p=0.5, tau=1, ema_beta=0.9, seed=seed, lookahead_delay=[1], **HP)
+    o2.init_params(0, w0)
+    tr = bruteforce.run(np.float32, R, N2, 0.5, 1, 0.9, HP["lr"], HP["beta1"], HP["beta2"], HP["eps"],
+                        HP["weight_decay"], seed, 5, w0, grads)
+    for t in range(4):
+        o2.step([grads[t]])
+        assert (o2.lookahead(0, 5).astype(np.float64) == tr[t]["look"]).all()
+
+
 # ---- P8: brute-force trace --------------------------------------------------------
 
 @pytest.mark.parametrize("tau,p,lam", [(2, 0.5, 0.9), (1, 0.3, 0.5), (0, 0.5, 0.9), (3, 1.0, 0.1)])
