@@ -17,11 +17,13 @@
 //   compact  slot = [cap][R]; a warp reserves room for its chunk's selected
 //            coordinates with one atomicAdd on the slot's cursor and records the
 //            base in chunk_base[slot][chunk]; tau steps later the consumer finds
-//            the data through that table and recomputes membership and rank
-//            from Philox, so no index list is stored.  tau + 1 slots.
+//            the data through that table and finds membership and rank again
+//            (this kernel from Philox, the pipelined one from the mask it stored
+//            with the slot), so no index list is stored.  tau / K + 1 slots
+//            (K: the averaging interval).
 //   dense    slot = [R][row_stride], replica-major like w, coordinate mu at position
 //            mu; used when the subset is so large that compaction saves nothing
-//            (d is replica-major too in this mode).  tau slots; the consumer and
+//            (d is replica-major too in this mode).  tau / K slots; the consumer and
 //            producer of a step share a slot and a thread reads a position
 //            before it overwrites it.
 // With tau = 0 (synchronous sparse averaging, Eq. "sparta") there is no ring:
