@@ -18,6 +18,9 @@
 //    drop the values those coordinates need (w^ and w^{t-1} per replica) into a
 //    small shared-memory stash; afterwards lane q finishes the q-th selected
 //    coordinate for all replicas with vector accesses to the ring and to d.
+//    (With 5 to 8 replicas the wide shape skips the value stash: the finishing
+//    lane reads w^{t-1} from the w rows before they are written and w^ from
+//    them afterwards.)
 //    Its ring and d loads are issued before the dense arithmetic starts, so
 //    their latency hides behind it.  Coordinates beyond the stash capacity
 //    (possible only for large p) are handled in place by their owning lane.
@@ -187,6 +190,14 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
     constexpr int NB = SH::kBits;   // mask bits per lane and sub-iteration
     constexpr int kUnitBytes = SH::kUnitBytes;
     constexpr int kPipeSubCoords = SH::kSubCoords;
+    // Wide shape, 5 to 8 replicas: the sparse phase takes w^ back from the w row the dense
+    // phase has just written (an L2 hit) and w^{t-1} from the same row before it is
+    // written, instead of from the stash that predicated stores in the dense loop fill.
+    // Measured on the 350M layout (R = 8): 16.5 against 17.1 ms per step at p = 0.05, 15.86
+    // against 15.77 at p = 0.01; no difference at R = 4 (1B layout); beyond 8 replicas the
+    // registers for w^{t-1} (CAP / 32 entries per lane) are not there.
+    constexpr bool kReload = (MODE == kCompact) && R > 4 && R <= 8 && CAP <= 64;
+    constexpr int kRounds = (CAP + 31) / 32;
     extern __shared__ __align__(16) unsigned char dyn_smem_all[];
     StageDesc *sd = reinterpret_cast<StageDesc *>(dyn_smem_all);
     unsigned char *dyn_smem = dyn_smem_all + pipe_table_bytes(P.S);
@@ -337,6 +348,26 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     load_replicas<R>(st.D + (uint64_t)e_coord * R, s_dd);
                 }
             }
+            // w^{t-1} of the adopted entries (only consumed ones need it), straight from
+            // the w rows, which still hold it at this point
+            float wprev[kReload ? kRounds : 1][R];
+            if constexpr (kReload) {
+#pragma unroll
+                for (int rr = 0; rr < kRounds; ++rr) {
+                    const uint32_t q = rr * 32 + lane;
+#pragma unroll
+                    for (int i = 0; i < R; ++i) wprev[rr][i] = 0.f;
+                    if (q < n_s && (rr == 0 || n_s > 32u)) {
+                        const uint32_t cc = rr == 0 ? e_coord : st_coord[q];
+                        const uint32_t ci = rr == 0 ? e_c : st_cidx[q];
+                        if (ci != kInvalidBase) {
+#pragma unroll
+                            for (int i = 0; i < R; ++i)
+                                wprev[rr][i] = __ldcg(st.W + (uint64_t)i * stride + cc);
+                        }
+                    }
+                }
+            }
 
             // ---- dense arithmetic, one replica (= one pipeline unit) at a time ----
             // (unrolled only for few replicas: beyond that the loop body no longer
@@ -372,7 +403,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     }
                 }
 
-                if (sm) {   // hand w^ and w^{t-1} of selected coordinates to the stash
+                if (!kReload && sm) {   // hand w^ and w^{t-1} of selected coordinates to the stash
 #pragma unroll
                     for (int j = 0; j < NB; ++j) {
                         if ((sm >> j) & 1u) {
@@ -433,7 +464,10 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
             __syncwarp();   // stash complete; dense stores ordered before the fix-ups below
 
             // ---- sparse phase: lane q finishes the q-th selected coordinate -------
-            for (uint32_t r0 = 0; r0 < n_s; r0 += 32) {
+#pragma unroll
+            for (int rr = 0; rr < kRounds; ++rr) {
+                const uint32_t r0 = rr * 32;
+                if (r0 >= n_s) break;
                 const uint32_t q = r0 + lane;
                 if (q < n_s) {
                     if (r0 != 0) {   // later rounds: loads were not issued ahead
@@ -446,7 +480,12 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         }
                     }
                     float wh[R];
-                    load_replicas<R>(st_what + q * R, wh);
+                    if constexpr (kReload) {
+#pragma unroll
+                        for (int i = 0; i < R; ++i) wh[i] = __ldcg(st.W + (uint64_t)i * stride + e_coord);
+                    } else {
+                        load_replicas<R>(st_what + q * R, wh);
+                    }
                     if constexpr (MODE == kSync) {
                         // Eq. "sparta": the selected coordinate takes the replica mean; the
                         // EMA state stays exactly zero (its sample is w^ - w^), hence mean + 0
@@ -466,7 +505,12 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     } else if (e_c != kInvalidBase) {
                         // Eq. "ema" + corrected averaging on S^{t-tau}
                         float wold[R];
-                        load_replicas<R>(st_wold + q * R, wold);
+                        if constexpr (kReload) {
+#pragma unroll
+                            for (int i = 0; i < R; ++i) wold[i] = wprev[rr][i];
+                        } else {
+                            load_replicas<R>(st_wold + q * R, wold);
+                        }
                         float a = on_wire<false>(P, s_old[0]);
 #pragma unroll
                         for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire<false>(P, s_old[i]));
