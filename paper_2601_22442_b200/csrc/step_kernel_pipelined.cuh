@@ -31,6 +31,8 @@
 // hand-over they need costs more than the issue slots they save, so the
 // per-thread form stays.
 #pragma once
+#include <type_traits>
+
 #include "step_kernel.cuh"
 
 namespace amk {
@@ -373,6 +375,11 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
             // (unrolled only for few replicas: beyond that the loop body no longer
             // fits the instruction cache and fetch stalls cost more than the
             // loop overhead saves)
+            // Two copies of the loop: the one that runs (no selected coordinate beyond the
+            // stash) carries no code for the in-place work, which otherwise sits, never
+            // executed, in the middle of the hottest instructions.
+            auto dense = [&](auto in_place_tag) {
+            constexpr bool kInPlace = decltype(in_place_tag)::value;
 #pragma unroll(R <= 4 ? R : 1)
             for (int i = 0; i < R; ++i) {
                 cp_async_wait<NST - 2>();
@@ -413,7 +420,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         }
                     }
                 }
-                if (om) {   // stash full: this lane does the sparse work itself
+                if (kInPlace && om) {   // stash full: this lane does the sparse work itself
 #pragma unroll
                     for (int j = 0; j < NB; ++j) {
                         if ((om >> j) & 1u) {
@@ -461,6 +468,9 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     }
                 }
             }
+            };
+            if (CAP < kPipeSubCoords && n_u > (uint32_t)CAP) dense(std::true_type{});
+            else dense(std::false_type{});
             __syncwarp();   // stash complete; dense stores ordered before the fix-ups below
 
             // ---- sparse phase: lane q finishes the q-th selected coordinate -------
