@@ -380,7 +380,8 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
             // executed, in the middle of the hottest instructions.
             auto dense = [&](auto in_place_tag) {
             constexpr bool kInPlace = decltype(in_place_tag)::value;
-#pragma unroll(R <= 4 ? R : 1)
+            constexpr int kUnroll = R <= 4 ? R : 1;
+#pragma unroll(kUnroll)
             for (int i = 0; i < R; ++i) {
                 cp_async_wait<NST - 2>();
                 issue_unit<R, SH>(pf, P, sd, stage_base + wr * kUnitBytes, lane, n_warps);
