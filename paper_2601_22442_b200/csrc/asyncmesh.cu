@@ -293,7 +293,10 @@ static int grid_for(uint64_t items, int threads)
 
 static KernelChoice pick_kernel(uint32_t R, int mode, int pipelined, bool general, uint32_t S)
 {
-    if (pipelined) return R <= 8 ? pick_pipelined_few(R, pipelined, S) : pick_pipelined_many(R, pipelined, S);
+    if (pipelined && R <= 8)
+        return general ? pick_pipelined_few_general(R, pipelined, S) : pick_pipelined_few_common(R, pipelined, S);
+    if (pipelined)
+        return general ? pick_pipelined_many_general(R, pipelined, S) : pick_pipelined_many_common(R, pipelined, S);
     if (R <= 8) return pick_direct_few(R, mode, general);
     return general ? pick_direct_many_general(R, mode) : pick_direct_many_common(R, mode);
 }
@@ -451,9 +454,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
             h->pipelined = 2;
     }
 
-    // E4M3 exchange and the eager estimate exist in the direct kernel only
+    // E4M3 exchange and the eager estimate: the kernels' general form
     const bool general = h->wire == 2u || h->correction == ASYNCMESH_CORRECTION_EAGER;
-    if (general) h->pipelined = 0;
 
     auto bail = [&](int code, const char *what) {
         release_all(h);

@@ -104,9 +104,10 @@ __device__ __forceinline__ void st_stream(float *p, const float (&x)[4])
 // quantisation study).  The average is formed in fp32; a replica's own
 // staleness sample keeps using its own unrounded value.
 // GEN selects the general form (also E4M3, also the eager estimate below); the
-// kernels of the common configurations are compiled without it: the pipelined
-// kernel's run time moves by several percent with a handful of extra instructions
-// in its sparse phase (measured: +7 % inline, +2 % as out-of-line calls).
+// kernels of the common configurations are compiled without it, as instantiations
+// of their own: the pipelined kernel's run time moves by several percent with a
+// handful of extra instructions in its sparse phase (measured: +7 % inline, +2 %
+// as out-of-line calls, although they never run in those configurations).
 template <bool GEN>
 __device__ __forceinline__ float on_wire(const StepParams &P, float x)
 {

@@ -177,10 +177,12 @@ __device__ __forceinline__ void issue_unit(UnitCursor &c, const StepParams &P, c
     cp_async_commit();   // always: keeps the group count in step with the unit count
 }
 
+// GEN: the general form of the sparse arithmetic (see on_wire), a separate set of
+// instantiations.
 // MODE is kCompact (tau >= 1: ring, d, bitmap) or kSync (tau = 0, Eq. "sparta": the
 // replica mean of the selected coordinates is formed from the stash itself; needs
 // a stash that holds a whole sub-iteration, i.e. the narrow shape).
-template <int R, int NST, class SH, int MODE>
+template <int R, int NST, class SH, int MODE, bool GEN>
 __global__ void __launch_bounds__(kPipeThreads, 2)
 asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
 {
@@ -431,16 +433,16 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                                 const uint64_t ce = (uint64_t)(cfirst + __popc(cm & below)) * R;
                                 float old[R];
                                 load_replicas<R>(ring_cons + ce, old);
-                                float a = on_wire<false>(P, old[0]);
+                                float a = on_wire<GEN>(P, old[0]);
 #pragma unroll
-                                for (int q = 1; q < R; ++q) a = __fadd_rn(a, on_wire<false>(P, old[q]));
+                                for (int q = 1; q < R; ++q) a = __fadd_rn(a, on_wire<GEN>(P, old[q]));
                                 const float abar = __fdiv_rn(a, P.Rf);
                                 float *dp = st.D + (mu0 + (uint64_t)(j >> 2) * 128 + (j & 3)) * R + i;
                                 float old_i = old[0];
 #pragma unroll
                                 for (int q = 1; q < R; ++q) old_i = (q == i) ? old[q] : old_i;
                                 const float diff = __fsub_rn(whj, old_i);
-                                const float dn = staleness<false>(P, *dp, diff);
+                                const float dn = staleness<GEN>(P, *dp, diff);
                                 *dp = dn;
                                 wn[j >> 2][j & 3] = __fadd_rn(abar, dn);
                             }
@@ -502,9 +504,9 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         // EMA state stays exactly zero (its sample is w^ - w^), hence mean + 0
                         float wold[R];
                         load_replicas<R>(st_wold + q * R, wold);
-                        float a = on_wire<false>(P, wh[0]);
+                        float a = on_wire<GEN>(P, wh[0]);
 #pragma unroll
-                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire<false>(P, wh[i]));
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire<GEN>(P, wh[i]));
                         const float wnew = __fadd_rn(__fdiv_rn(a, P.Rf), 0.0f);
 #pragma unroll
                         for (int i = 0; i < R; ++i) {
@@ -522,14 +524,14 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         } else {
                             load_replicas<R>(st_wold + q * R, wold);
                         }
-                        float a = on_wire<false>(P, s_old[0]);
+                        float a = on_wire<GEN>(P, s_old[0]);
 #pragma unroll
-                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire<false>(P, s_old[i]));
+                        for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire<GEN>(P, s_old[i]));
                         const float abar = __fdiv_rn(a, P.Rf);
 #pragma unroll
                         for (int i = 0; i < R; ++i) {
                             const float diff = __fsub_rn(wh[i], s_old[i]);
-                            const float dn = staleness<false>(P, s_dd[i], diff);
+                            const float dn = staleness<GEN>(P, s_dd[i], diff);
                             s_dd[i] = dn;
                             const float wnew = __fadd_rn(abar, dn);
                             const uint64_t o1 = (uint64_t)i * stride + e_coord;

@@ -1,10 +1,11 @@
-// Instantiations of the step kernels.  Compiled five times, -DAM_PART=0..4:
+// Instantiations of the step kernels.  Compiled seven times, -DAM_PART=0..6:
 // 0 direct kernel R = 1..8; 1 direct kernel R = 9..16, common form; 2 the same,
-// general form; 3 pipelined kernel R = 1..8; 4 pipelined kernel R = 9..16.
+// general form; 3 / 4 pipelined kernel R = 1..8, common / general form; 5 / 6
+// pipelined kernel R = 9..16, common / general form.
 #include "kernel_table.cuh"
 
 #ifndef AM_PART
-#error "compile with -DAM_PART=0..4"
+#error "compile with -DAM_PART=0..6"
 #endif
 
 namespace amk {
@@ -67,11 +68,13 @@ KernelChoice pick_direct_many_general(uint32_t R, int mode)
 
 #else   // pipelined kernel
 
+constexpr bool kGeneral = (AM_PART == 4 || AM_PART == 6);
+
 template <int R, class SH, int MODE>
 static KernelChoice pipelined_as(uint32_t S)
 {
     KernelChoice c;
-    c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, SH, MODE>;
+    c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, SH, MODE, kGeneral>;
     c.threads = kPipeThreads;
     c.smem = (size_t)pipe_table_bytes(S) +
              (size_t)(kPipeThreads / 32) * PipeCfg<R, SH>::warp_bytes(kPipeStages);
@@ -90,9 +93,17 @@ static KernelChoice pipelined(int shape, uint32_t S)
 }
 
 #if AM_PART == 3
-KernelChoice pick_pipelined_few(uint32_t R, int shape, uint32_t S)
+KernelChoice pick_pipelined_few_common(uint32_t R, int shape, uint32_t S)
+#elif AM_PART == 4
+KernelChoice pick_pipelined_few_general(uint32_t R, int shape, uint32_t S)
+#elif AM_PART == 5
+KernelChoice pick_pipelined_many_common(uint32_t R, int shape, uint32_t S)
+#else
+KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S)
+#endif
 {
     switch (R) {
+#if AM_PART <= 4
     case 1: return pipelined<1>(shape, S);
     case 2: return pipelined<2>(shape, S);
     case 3: return pipelined<3>(shape, S);
@@ -101,13 +112,7 @@ KernelChoice pick_pipelined_few(uint32_t R, int shape, uint32_t S)
     case 6: return pipelined<6>(shape, S);
     case 7: return pipelined<7>(shape, S);
     case 8: return pipelined<8>(shape, S);
-    default: return KernelChoice();
-    }
-}
 #else
-KernelChoice pick_pipelined_many(uint32_t R, int shape, uint32_t S)
-{
-    switch (R) {
     case 9: return pipelined<9>(shape, S);
     case 10: return pipelined<10>(shape, S);
     case 11: return pipelined<11>(shape, S);
@@ -116,10 +121,10 @@ KernelChoice pick_pipelined_many(uint32_t R, int shape, uint32_t S)
     case 14: return pipelined<14>(shape, S);
     case 15: return pipelined<15>(shape, S);
     case 16: return pipelined<16>(shape, S);
+#endif
     default: return KernelChoice();
     }
 }
-#endif
 
 #endif
 
