@@ -27,7 +27,7 @@ def slices_for(n):
     return [(0, SLICE)] + [(m, SLICE) for m in mids] + [(n - SLICE, SLICE)]
 
 
-def run_full(R, numel, p, tau, steps, lam=0.9):
+def run_full(R, numel, p, tau, steps, lam=0.9, extra_slices=()):
     import paper_2601_22442_b200 as pkg
     from paper_2601_22442_b200.layouts import DEFAULT_HP
     hp = dict(DEFAULT_HP, p=p, ema_beta=lam)
@@ -38,7 +38,7 @@ def run_full(R, numel, p, tau, steps, lam=0.9):
             pytest.skip("not enough free device memory for R=%d p=%g tau=%d" % (R, p, tau))
         raise
     dev = torch.device("cuda", 0)
-    sl = [slices_for(n) for n in numel]
+    sl = [slices_for(n) + [(b, SLICE) for b in extra_slices] for n in numel]
     oracles = []   # one oracle per slice index; its stages are that slice of every stage
     n_slices = max(len(x) for x in sl)
     for k in range(n_slices):
@@ -113,3 +113,19 @@ def test_config_llama1b_20_steps():
 def test_config_sweep_on_350m_layout(p, tau):
     w = workloads()["llama350m"]
     run_full(w["R"], w["numel"], p, tau, 20)
+
+
+@pytest.mark.parametrize("R,n,p,tau", [
+    (1, 2 ** 32 - 1 - 37, 0.05, 2),      # the largest stage the interface takes (ragged: not a multiple of 4)
+    (2, 2 ** 31 + 4096 + 5, 0.05, 1),    # second replica row starts beyond 2^31 floats, ends beyond 2^32
+    (2, 2 ** 31 + 4096 + 5, 1.0, 1),     # the same through the dense ring
+])
+def test_maximum_stage_sizes(R, n, p, tau):
+    # 64-bit offsets everywhere: ~100 GB of state in one stage, slices at both ends, at thirds,
+    # across coordinate 2^31 and across the last warp chunk
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    need = (5 + (tau if p == 1.0 else 0)) * R * n * 4 + (6 << 30)
+    if free < need:
+        pytest.skip("needs %.0f GB of free device memory, %.0f GB are free" % (need / 1e9, free / 1e9))
+    run_full(R, [n], p, tau, 2 * tau + 3, extra_slices=(2 ** 31 - 1500, n - 4000))
