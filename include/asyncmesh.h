@@ -133,9 +133,11 @@ typedef struct asyncmesh_config {
 /*
  * Create the state: per stage W, M, V (replica-major rows [R][row_stride]),
  * D (coordinate-major [row_stride][R]; replica-major with the dense ring), LOOK
- * (only where delta_j > 0) and the snapshot ring (compact: room for the selected
- * coordinates only, tau + 1 slots; dense, for large p: one position per
- * coordinate and replica, tau slots).  The library owns all of it (obtained through cfg->alloc).
+ * (only where delta_j > 0), a copy of the previous weights (only with
+ * ASYNCMESH_FLAG_KEEP_PREVIOUS) and the snapshot ring (compact: room for the
+ * selected coordinates only, tau / K + 1 slots; dense, for large p: one position
+ * per coordinate and replica, tau / K slots; K = avg_interval).  The library owns
+ * all of it (obtained through cfg->alloc).
  * Moments, D and the ring start at zero, the step counter at 0, weights are
  * unset until asyncmesh_init_params.  The config and its arrays are copied.
  * Errors: INVALID_ARG (range checks above), OOM (allocator returned NULL: every

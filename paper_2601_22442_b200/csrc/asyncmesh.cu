@@ -92,7 +92,7 @@ struct asyncmesh {
     StageDesc *sd_dev = nullptr;
     unsigned int *cursors = nullptr;  // [n_slots][S]
     int *status = nullptr;
-    double *scratch = nullptr;        // one double for reductions
+    double *scratch = nullptr;        // a few doubles for reductions
 
     int mode = kSync;
     int pipelined = 0;
