@@ -128,6 +128,14 @@ typedef struct asyncmesh_config {
     uint32_t correction;             /* ASYNCMESH_CORRECTION_EMA (0) or ASYNCMESH_CORRECTION_EAGER */
     double momentum_decay;           /* NAdamW: psi of mu_t = beta1 (1 - 0.5 * 0.96^(t psi));
                                         0 selects the customary 0.004                   */
+    const uint64_t *coord_base;      /* host [S] or NULL (all 0): global index of this handle's
+                                        coordinate 0 of stage j, when the handle holds one
+                                        coordinate range of a larger stage (a shard; coordinates
+                                        are independent of one another, Appendix A, so ranges of
+                                        a stage can live on different GPUs with no exchange).
+                                        The subset rule uses the global index, so shards select
+                                        exactly what the unsharded stage would.  Multiples of 4;
+                                        coord_base + stage_numel <= 2^32                 */
 } asyncmesh_config;
 
 /*

@@ -48,6 +48,7 @@ class Config(ctypes.Structure):
         ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_ctx", ctypes.c_void_p),
         ("optimizer", ctypes.c_uint32), ("correction", ctypes.c_uint32),
         ("momentum_decay", ctypes.c_double),
+        ("coord_base", ctypes.POINTER(ctypes.c_uint64)),
     ]
 
 
@@ -159,7 +160,7 @@ class AsyncMesh:
                  allocator: Optional[TorchAllocator] = None,
                  use_torch_allocator: bool = True, flags: int = 0, avg_interval: int = 1,
                  optimizer: str = "adamw", momentum_decay: float = 4e-3,
-                 correction: str = "ema"):
+                 correction: str = "ema", coord_base: Optional[Sequence[int]] = None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("asyncmesh needs a CUDA device; there is no CPU path")
@@ -188,6 +189,9 @@ class AsyncMesh:
         cfg.device, cfg.avg_interval, cfg.stream = self.device, int(avg_interval), stream
         cfg.optimizer = {"adamw": 0, "nadamw": 1}[optimizer]
         cfg.correction = {"ema": 0, "eager": 1}[correction]
+        if coord_base is not None:
+            self._base = (ctypes.c_uint64 * self.S)(*[int(b) for b in coord_base])
+            cfg.coord_base = self._base
         cfg.momentum_decay = float(momentum_decay)
         if self.allocator is not None:
             cfg.alloc, cfg.free = self.allocator.alloc_cb, self.allocator.free_cb

@@ -141,14 +141,14 @@ static void release_all(asyncmesh *h)
 // ---------------------------------------------------------------------------
 
 __global__ void subset_bitmap_kernel(SubsetRule rule, uint32_t stage, uint32_t step, uint64_t N,
-                                     uint8_t *bitmap)
+                                     uint32_t quad_base, uint8_t *bitmap)
 {
     const uint64_t nbytes = (N + 7) / 8;
     for (uint64_t b = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nbytes;
          b += (uint64_t)gridDim.x * blockDim.x) {
         const uint64_t mu = b * 8;
-        uint32_t bits = subset_bits(rule, stage, step, (uint32_t)(mu >> 2));
-        if (mu + 4 < N) bits |= subset_bits(rule, stage, step, (uint32_t)((mu + 4) >> 2)) << 4;
+        uint32_t bits = subset_bits(rule, stage, step, quad_base + (uint32_t)(mu >> 2));
+        if (mu + 4 < N) bits |= subset_bits(rule, stage, step, quad_base + (uint32_t)((mu + 4) >> 2)) << 4;
         const uint64_t left = N - mu;
         if (left < 8) bits &= (1u << (uint32_t)left) - 1u;
         bitmap[b] = (uint8_t)bits;
@@ -361,6 +361,12 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     for (uint32_t s = 0; s < cfg->S; ++s)
         if (cfg->stage_numel[s] < 1 || cfg->stage_numel[s] > 0xFFFFFFFFull)
             return fail(ASYNCMESH_ERR_INVALID_ARG, "create: stage_numel[%u] outside 1..2^32-1", s);
+    if (cfg->coord_base)
+        for (uint32_t s = 0; s < cfg->S; ++s)
+            if ((cfg->coord_base[s] & 3u) != 0 || cfg->coord_base[s] + cfg->stage_numel[s] > 0x100000000ull)
+                return fail(ASYNCMESH_ERR_INVALID_ARG,
+                            "create: coord_base[%u] must be a multiple of 4 and coord_base + stage_numel "
+                            "at most 2^32", s);
 
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
@@ -475,8 +481,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         d.N = h->numel[s];
         d.stride = h->stride[s];
         d.stage_id = s;
+        d.quad_base = cfg->coord_base ? (uint32_t)(cfg->coord_base[s] >> 2) : 0u;
         d.delta = (float)h->delay[s];
-        d.has_look = h->delay[s] != 0 ? 1u : 0u;
         d.cap = (uint32_t)cap[s];
         d.W = (float *)zalloc(row_bytes);
         d.M = (float *)zalloc(row_bytes);
@@ -488,7 +494,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
             if (!h->wprev[s]) return bail(ASYNCMESH_ERR_OOM, "out of device memory (previous weights)");
         }
         d.LOOK = d.W;
-        if (d.has_look) {
+        if (h->delay[s] != 0) {
             d.LOOK = (float *)zalloc(row_bytes);
             if (!d.LOOK) return bail(ASYNCMESH_ERR_OOM, "out of device memory (look-ahead)");
         }
@@ -581,7 +587,7 @@ extern "C" int asyncmesh_init_params(asyncmesh *h, uint32_t stage, int32_t repli
     for (uint32_t i = 0; i < h->R; ++i) {
         if (replica >= 0 && (uint32_t)replica != i) continue;
         CU_TRY(cudaMemcpyAsync(d.W + (uint64_t)i * d.stride, src, n * sizeof(float), kind, h->stream));
-        if (d.has_look)
+        if (d.LOOK != d.W)
             CU_TRY(cudaMemcpyAsync(d.LOOK + (uint64_t)i * d.stride, src, n * sizeof(float), kind,
                                    h->stream));
     }
@@ -864,7 +870,8 @@ extern "C" int asyncmesh_subset_mask(asyncmesh *h, uint32_t stage, uint64_t step
     const uint64_t N = h->numel[stage], nbytes = (N + 7) / 8;
     uint8_t *tmp = (uint8_t *)dev_alloc(h, nbytes);
     if (!tmp) return fail(ASYNCMESH_ERR_OOM, "subset_mask: out of device memory (temporary)");
-    subset_bitmap_kernel<<<grid_for(nbytes, 256), 256, 0, h->stream>>>(h->rule, stage, (uint32_t)step, N, tmp);
+    subset_bitmap_kernel<<<grid_for(nbytes, 256), 256, 0, h->stream>>>(h->rule, stage, (uint32_t)step, N,
+                                                                          h->sd[stage].quad_base, tmp);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) e = cudaMemcpyAsync(bitmap_host, tmp, nbytes, cudaMemcpyDeviceToHost, h->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);

@@ -66,8 +66,9 @@ struct StageDesc {
     uint32_t chunk_begin;   // first chunk of this stage in the global list
     uint32_t cap;           // selected coordinates a compact slot can hold
     uint32_t stage_id;
-    float delta;            // look-ahead delay as a float
-    uint32_t has_look;      // LOOK is a buffer of its own
+    float delta;            // look-ahead delay as a float; != 0: LOOK is a buffer of its own
+    uint32_t quad_base;     // (global index of local coordinate 0) / 4: a handle may hold a
+                            // coordinate range of a larger stage (one shard per GPU)
 };
 
 struct StepParams {
@@ -205,7 +206,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
         if (mu < N) {
             const uint64_t left = N - mu;
             const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
-            const uint32_t quad = (uint32_t)(mu >> 2);
+            const uint32_t quad = st.quad_base + (uint32_t)(mu >> 2);
             if (P.produce)
                 pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * k);
             if (consume)
@@ -242,7 +243,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
     const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
     float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
     const float delta = st.delta;
-    const bool has_look = st.has_look != 0u;
+    const bool has_look = st.delta != 0.0f;
 
 #pragma unroll 1
     for (int k = 0; k < kSubIters; ++k) {

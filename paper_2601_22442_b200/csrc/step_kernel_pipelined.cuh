@@ -108,7 +108,9 @@ struct PipeCfg {
 // Dynamic shared memory: the stage table (S entries), then one region per warp.
 __host__ __device__ constexpr int pipe_table_bytes(uint32_t S)
 {
-    return (int)((S * sizeof(StageDesc) + 15) / 16 * 16);
+    // a multiple of 128 bytes: the warps' copy stages behind it then start on a 128-byte
+    // boundary, and a warp's 512-byte rows of 16-byte copies fall into whole shared-memory lines
+    return (int)((S * sizeof(StageDesc) + 127) / 128 * 128);
 }
 
 template <class SH>
@@ -260,13 +262,14 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         // above: the generator runs once per coordinate and step) ----
         // bit 4b + c  <->  coordinate c0 + 128 b + c; sub-iteration k owns bits NB*k ..
         uint32_t pmask = 0;
+        const uint32_t quad0 = st.quad_base + (uint32_t)(c0 >> 2);   // global index / 4 of the lane's first quad
 #pragma unroll 2
         for (int b = 0; b < 8; ++b) {   // 8 quads per lane and chunk
             const uint64_t mu = c0 + (uint64_t)b * 128;
             if (mu < N) {
                 const uint64_t left = N - mu;
                 const uint32_t valid = left >= 4 ? 0xFu : ((1u << (uint32_t)left) - 1u);
-                const uint32_t quad = (uint32_t)(mu >> 2);
+                const uint32_t quad = quad0 + (uint32_t)b * 32u;
                 if (P.produce)
                     pmask |= (subset_bits(P.rule, st.stage_id, P.step, quad) & valid) << (4 * b);
             }
@@ -302,7 +305,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
         float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
         const float delta = st.delta;
-        const bool has_look = st.has_look != 0u;
+        const bool has_look = st.delta != 0.0f;
 
 #pragma unroll 1
         for (int k = 0; k < kmax; ++k) {

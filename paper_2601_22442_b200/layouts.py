@@ -6,7 +6,7 @@ pipeline stages (Section 2.1: P stages, each a contiguous run of layers).
 """
 from __future__ import annotations
 
-from typing import Dict, List
+from typing import Dict, List, Sequence
 
 
 def llama_stage_numel(d: int, layers: int, ffn: int, vocab: int, stages: int,
@@ -21,6 +21,31 @@ def llama_stage_numel(d: int, layers: int, ffn: int, vocab: int, stages: int,
     out[0] += vocab * d
     out[-1] += d + (0 if tied else vocab * d)
     return out
+
+
+def coordinate_shard(numel: Sequence[int], rank: int, world: int, align: int = 1024):
+    """The coordinate range of every stage that shard ``rank`` of ``world`` holds.
+
+    Coordinates are independent of one another (Appendix A, remark after Theorem 2)
+    and the replica average runs over rows that live together, so a stage can be
+    cut into ranges that live on different GPUs with no exchange at all.  Returns
+    (shard_numel, coord_base): stage j's shard is [coord_base[j], coord_base[j] +
+    shard_numel[j]); the cuts are multiples of ``align`` (itself a multiple of 4,
+    which the subset rule needs) and the ranges tile the stage exactly.  A stage
+    with fewer than ``world`` aligned pieces cannot be cut that far: ValueError.
+    """
+    if align % 4 or not (0 <= rank < world):
+        raise ValueError("align must be a multiple of 4 and 0 <= rank < world")
+    sizes, bases = [], []
+    for n in numel:
+        pieces = (int(n) + align - 1) // align                 # aligned pieces, the last one ragged
+        if pieces < world:
+            raise ValueError("a stage of %d coordinates has fewer than %d pieces of %d" % (n, world, align))
+        lo = (pieces * rank // world) * align
+        hi = min((pieces * (rank + 1) // world) * align, int(n))
+        sizes.append(max(hi - lo, 0))
+        bases.append(min(lo, int(n)))
+    return sizes, bases
 
 
 # The benchmark configurations (R replicas, stage sizes, delay tau, steps).

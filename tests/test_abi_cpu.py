@@ -44,7 +44,7 @@ def test_config_struct_matches_header_layout():
     assert offs["device"] == 96 and offs["avg_interval"] == 100 and offs["stream"] == 104
     assert offs["alloc"] == 112 and offs["free"] == 120 and offs["alloc_ctx"] == 128
     assert offs["optimizer"] == 136 and offs["correction"] == 140 and offs["momentum_decay"] == 144
-    assert ctypes.sizeof(binding.Config) == 152
+    assert offs["coord_base"] == 152 and ctypes.sizeof(binding.Config) == 160
 
 
 def _cfg(**over):
@@ -67,6 +67,8 @@ def _cfg(**over):
     (dict(eps=0.0), "eps"), (dict(beta1=1.0), "betas"), (dict(tau=3, avg_interval=2), "avg_interval"),
     (dict(avg_interval=-1), "avg_interval"), (dict(optimizer=2), "optimizer"), (dict(flags=8), "flags"), (dict(flags=256), "flags"),
     (dict(flags=16 | 64), "exclude"), (dict(correction=2), "correction"),
+    (dict(coord_base=(ctypes.c_uint64 * 1)(6)), "coord_base"),
+    (dict(coord_base=(ctypes.c_uint64 * 1)(2 ** 32 - 4)), "coord_base"),
 ])
 def test_create_rejects_bad_arguments_without_touching_a_device(lib, over, word):
     h = ctypes.c_void_p()

@@ -6,6 +6,9 @@ import socket
 import subprocess
 import sys
 
+import pytest
+import torch
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -72,3 +75,40 @@ def test_single_rank_aggregation_is_identity():
     import bench
     assert bench.aggregate_over_ranks(3.5, 7.0, 1) == (3.5, 7.0)
     assert bench.measured_peak_gbs()[0] > 1000
+
+
+def _shard_worker(rank, world, port, numel, out):
+    import torch.distributed as dist
+    from paper_2601_22442_b200.layouts import coordinate_shard
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    sizes, bases = coordinate_shard(numel, rank, world)
+    mine = torch.tensor([sizes, bases], dtype=torch.int64)
+    gathered = [torch.zeros_like(mine) for _ in range(world)]
+    dist.all_gather(gathered, mine)          # host-side bookkeeping only: the data path has no collective
+    if rank == 0:
+        out.put([g.tolist() for g in gathered])
+    dist.destroy_process_group()
+
+
+def test_coordinate_shards_of_two_ranks_tile_every_stage():
+    import multiprocessing as mp
+    from paper_2601_22442_b200.layouts import coordinate_shard, workloads
+    numel = workloads()["llama125m"]["numel"] + [4099]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = free_port()
+    procs = [ctx.Process(target=_shard_worker, args=(r, 2, port, numel, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (s0, b0), (s1, b1) = got
+    for j, n in enumerate(numel):
+        assert b0[j] == 0 and b1[j] == s0[j] and s0[j] + s1[j] == n     # exact tiling, in order
+        assert b1[j] % 1024 == 0 and s0[j] > 0 and s1[j] > 0
+    with pytest.raises(ValueError):
+        coordinate_shard([1000], 0, 2)
+    with pytest.raises(ValueError):
+        coordinate_shard([5000], 0, 2, align=6)

@@ -352,6 +352,42 @@ def test_lookahead_for_any_delay_with_kept_previous_weights(p, tau):
     assert g.lookahead_weights(0, 2)[0] != g.lookahead_weights(0, 7)[0]   # configured delay: the fused buffer
 
 
+@pytest.mark.parametrize("p,tau,flags", [(0.05, 2, 0), (0.3, 1, 0), (1.0, 1, 0), (0.3, 0, 0), (0.2, 1, 2)])
+def test_coordinate_shards_equal_the_unsharded_stage(p, tau, flags):
+    # two handles, each with one coordinate range of every stage (what two GPUs would hold),
+    # against the oracle of the whole stage: same subsets (global index in the rule), same state
+    from paper_2601_22442_b200.layouts import coordinate_shard
+    R, numel, steps = 3, [9000, 4096 + 77], 2 * tau + 4
+    o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=0.9, **HP)
+    for s, n in enumerate(numel):
+        o.init_params(s, si.init_weights_host(0x1217, s, 0, n))
+    shards = []
+    for rank in range(2):
+        sizes, bases = coordinate_shard(numel, rank, 2)
+        g = am().AsyncMesh(R, sizes, p=p, tau=tau, ema_beta=0.9, flags=flags, coord_base=bases,
+                           lookahead_delay=[1, 0], **HP)
+        for s in range(2):
+            g.init_params(s, si.init_weights_host(0x1217, s, bases[s], sizes[s]))
+        shards.append((g, sizes, bases, g.empty_grads()))
+    o2 = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=0.9, lookahead_delay=[1, 0], **HP)
+    for s, n in enumerate(numel):
+        o2.init_params(s, si.init_weights_host(0x1217, s, 0, n))
+    for t in range(1, steps + 1):
+        o2.step([si.grads_host(0x6AD5, t, s, R, 0, n) for s, n in enumerate(numel)])
+        for g, sizes, bases, bufs in shards:
+            for s in range(2):
+                bufs[s][:, :sizes[s]].copy_(torch.from_numpy(si.grads_host(0x6AD5, t, s, R, bases[s], sizes[s])))
+            g.step(bufs)
+    for s, n in enumerate(numel):
+        for name in STATE_NAMES:
+            whole = np.concatenate([g.get(s, name) for g, _, _, _ in shards], axis=1)
+            assert np.array_equal(whole, o2.get(s, name)), (s, name)
+        mask = np.concatenate([g.subset_mask(s, steps) for g, _, _, _ in shards])
+        assert np.array_equal(mask, o2.subset_mask(s, steps))
+    with pytest.raises(am().AsyncMeshError):
+        am().AsyncMesh(R, [100], p=p, tau=tau, ema_beta=0.9, coord_base=[6], **HP)
+
+
 def test_step_host_equals_step():
     numel = [3000, 1025]
     a = am().AsyncMesh(3, numel, p=0.2, tau=1, ema_beta=0.9, **HP)
