@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--flags", type=int, default=0, help="asyncmesh_config.flags (diagnostic)")
+    ap.add_argument("--optimizer", choices=["adamw", "nadamw"], default="adamw",
+                    help="diagnostic: the paper's own NAdamW instead of the workloads' AdamW")
     return ap.parse_args()
 
 
@@ -216,7 +218,9 @@ def run_reference(args):
 def config_dict(args, w, hp):
     return {"workload": args.workload, "R": w["R"], "S": len(w["numel"]),
             "params_per_replica": sum(w["numel"]), "p": hp["p"], "tau": w["tau"],
-            "ema_beta": hp["ema_beta"], "optimizer": "AdamW lr=3e-4 (0.9,0.95) wd=0.1 eps=1e-8",
+            "ema_beta": hp["ema_beta"],
+            "optimizer": ("NAdamW" if getattr(args, "optimizer", "adamw") == "nadamw" else "AdamW")
+            + " lr=3e-4 (0.9,0.95) wd=0.1 eps=1e-8",
             "lookahead_delay": "S-1-stage", "state": "fp32",
             "l2": "inputs larger than L2 (every step streams the whole state)"}
 
@@ -250,7 +254,7 @@ def run_native(args):
     mesh = pkg.AsyncMesh(R, numel, p=hp["p"], tau=tau, ema_beta=hp["ema_beta"], lr=hp["lr"],
                          beta1=hp["beta1"], beta2=hp["beta2"], eps=hp["eps"],
                          weight_decay=hp["weight_decay"], seed=MESH_SEED + rank, device=local,
-                         stream=stream.cuda_stream, flags=args.flags)
+                         stream=stream.cuda_stream, flags=args.flags, optimizer=args.optimizer)
     for s, n in enumerate(numel):
         tmp = torch.empty(n, dtype=torch.float32, device=dev)
         si.normal_device(tmp, si.stream_key(INIT_SEED + rank, si.KIND_INIT, 0, s, 0), 0, 0.02)
