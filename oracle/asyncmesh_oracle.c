@@ -62,7 +62,11 @@
  * against torch.optim.AdamW and a closed form, the reductions tau=0 -> Eq.
  * "sparta", lambda=0 -> Eq. "asparta", lambda=1 -> raw difference, p=1,tau=0
  * -> full averaging, mean invariance, Lemma 1's (1-p) factor, a brute-force
- * trace written separately from the equations, chunk independence.
+ * trace written separately from the equations (also with an averaging interval,
+ * with the bfloat16 / E4M3 exchange and with the eager estimate), chunk
+ * independence; NAdamW against torch.optim.NAdam; the bfloat16 and E4M3 roundings
+ * against the formats' definitions and the tensor library's casts; the eager
+ * estimate against its closed form; the spread of d against numpy.
  * The look-ahead formula for delay > 0 is this build's reading of a sentence
  * (the paper prints no formula): PARITY UNPINNED beyond delay = 0 and the
  * constant-velocity closed form.
