@@ -204,6 +204,11 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
     // registers for w^{t-1} (CAP / 32 entries per lane) are not there.
     constexpr bool kReload = (MODE == kCompact) && R > 4 && R <= 8 && CAP <= 64;
     constexpr int kRounds = (CAP + 31) / 32;
+    // rounds of the sparse phase whose ring and d loads go out before the dense loop; the
+    // narrow shape serves subsets for which a second round is the rule, not the exception
+    // (1B layout, R = 4, p = 0.25: 31.1 -> 29.9 ms; with 8 replicas the registers this
+    // takes cost more than it saves: 20.4 -> 21.1 ms on the 350M layout)
+    constexpr int kPre = (V == 1 && MODE == kCompact && R <= 4) ? 2 : 1;
     extern __shared__ __align__(16) unsigned char dyn_smem_all[];
     StageDesc *sd = reinterpret_cast<StageDesc *>(dyn_smem_all);
     unsigned char *dyn_smem = dyn_smem_all + pipe_table_bytes(P.S);
@@ -355,6 +360,22 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     load_replicas<R>(st.D + (uint64_t)e_coord * R, s_dd);
                 }
             }
+            // a second entry per lane when the subset is large
+            uint32_t e1_coord = 0, e1_c = kInvalidBase, e1_p = kInvalidBase;
+            float s1_old[kPre > 1 ? R : 1], s1_dd[kPre > 1 ? R : 1];
+            if constexpr (kPre > 1) {
+#pragma unroll
+                for (int i = 0; i < R; ++i) { s1_old[i] = 0.f; s1_dd[i] = 0.f; }
+                if (32u + (uint32_t)lane < n_s) {
+                    e1_coord = st_coord[32 + lane];
+                    e1_c = st_cidx[32 + lane];
+                    e1_p = st_pidx[32 + lane];
+                    if (e1_c != kInvalidBase) {
+                        load_replicas<R>(ring_cons + (uint64_t)e1_c * R, s1_old);
+                        load_replicas<R>(st.D + (uint64_t)e1_coord * R, s1_dd);
+                    }
+                }
+            }
             // w^{t-1} of the adopted entries (only consumed ones need it), straight from
             // the w rows, which still hold it at this point
             float wprev[kReload ? kRounds : 1][R];
@@ -486,7 +507,13 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                 if (r0 >= n_s) break;
                 const uint32_t q = r0 + lane;
                 if (q < n_s) {
-                    if (r0 != 0) {   // later rounds: loads were not issued ahead
+                    if (kPre > 1 && rr == 1) {   // second round: asked for ahead as well
+                        e_coord = e1_coord;
+                        e_c = e1_c;
+                        e_p = e1_p;
+#pragma unroll
+                        for (int i = 0; i < R; ++i) { s_old[i] = s1_old[i]; s_dd[i] = s1_dd[i]; }
+                    } else if (r0 != 0) {   // later rounds: loads were not issued ahead
                         e_coord = st_coord[q];
                         e_c = st_cidx[q];
                         e_p = st_pidx[q];
