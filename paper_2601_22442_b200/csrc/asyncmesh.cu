@@ -550,6 +550,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         delete h;
         return fail(ASYNCMESH_ERR_CUDA, "create: the step kernel cannot run on this device: %s", msg);
     }
+    if (h->kernel.max_blocks_per_sm > 0 && per_sm > h->kernel.max_blocks_per_sm)
+        per_sm = h->kernel.max_blocks_per_sm;
     uint64_t blocks = (uint64_t)sms * per_sm;
     const uint64_t wpb = (uint64_t)h->kernel.threads / 32;
     const uint64_t need = ((uint64_t)h->total_chunks + wpb - 1) / wpb;

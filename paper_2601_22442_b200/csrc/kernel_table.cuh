@@ -13,6 +13,7 @@ struct KernelChoice {
     step_fn fn = nullptr;
     size_t smem = 0;              // dynamic shared memory per block
     int threads = kBlockThreads;  // block size
+    int max_blocks_per_sm = 0;    // 0: as many as fit
 };
 
 // general: the form that also knows the E4M3 exchange and the eager staleness

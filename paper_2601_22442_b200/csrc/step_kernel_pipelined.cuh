@@ -37,7 +37,11 @@
 
 namespace amk {
 
-constexpr int kPipeThreads = 192;   // 6 warps; 2 blocks per SM
+constexpr int kPipeThreads = 128;   // 4 warps per block
+constexpr int kPipeBlocksPerSM = 3; // at most: 12 warps per SM.  Measured on the 1B layout: 10 warps 24.9 ms,
+                                    // 12 warps 23.6, 14 warps 23.9, 18 warps 25.9; with 8 replicas the wide
+                                    // shape takes more registers than three blocks leave and runs 8 warps
+                                    // (350M layout 15.8 ms against 16.3 for 12 warps held to 156 registers)
 constexpr int kPipeStages = 3;      // units in the shared-memory ring of a warp
 
 // Two shapes of the same kernel.  Wide: 8 coordinates per lane and unit, stash

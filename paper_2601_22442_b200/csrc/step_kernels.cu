@@ -76,6 +76,7 @@ static KernelChoice pipelined_as(uint32_t S)
     KernelChoice c;
     c.fn = asyncmesh_step_kernel_pipelined<R, kPipeStages, SH, MODE, kGeneral>;
     c.threads = kPipeThreads;
+    c.max_blocks_per_sm = kPipeBlocksPerSM;
     c.smem = (size_t)pipe_table_bytes(S) +
              (size_t)(kPipeThreads / 32) * PipeCfg<R, SH>::warp_bytes(kPipeStages);
     return c;
