@@ -64,6 +64,9 @@ extern "C" {
                                           where the shared-memory pipelined one applies  */
 #define ASYNCMESH_FLAG_PIPELINED_KERNEL 4u /* use the compact ring and the pipelined kernel for
                                              any p (diagnostic: exercises its in-place path) */
+#define ASYNCMESH_FLAG_OWNER_KERNEL 256u /* use the kernel in which the lane that owns a coordinate
+                                           does all of its work (up to four replicas, compact ring
+                                           or tau = 0) */
 #define ASYNCMESH_FLAG_BF16_EXCHANGE 16u /* the subset is exchanged in bfloat16 (the paper's
                                            quantisation study): every snapshot value entering the
                                            replica average is first rounded to bfloat16 (nearest

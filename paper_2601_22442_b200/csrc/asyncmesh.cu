@@ -293,6 +293,10 @@ static int grid_for(uint64_t items, int threads)
 
 static KernelChoice pick_kernel(uint32_t R, int mode, int pipelined, bool general, uint32_t S)
 {
+    if (pipelined >= 4) {
+        const int entries = pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany;
+        return general ? pick_owner_general(R, mode, entries, S) : pick_owner_common(R, mode, entries, S);
+    }
     if (pipelined && R <= 8)
         return general ? pick_pipelined_few_general(R, pipelined, S) : pick_pipelined_few_common(R, pipelined, S);
     if (pipelined)
@@ -346,7 +350,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
                         ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE |
                         ASYNCMESH_FLAG_DENSE_RING | ASYNCMESH_FLAG_FP8_EXCHANGE |
-                        ASYNCMESH_FLAG_KEEP_PREVIOUS)) != 0)
+                        ASYNCMESH_FLAG_KEEP_PREVIOUS | ASYNCMESH_FLAG_OWNER_KERNEL)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
     if ((cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) && (cfg->flags & ASYNCMESH_FLAG_FP8_EXCHANGE))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: BF16_EXCHANGE and FP8_EXCHANGE exclude each other");
@@ -446,13 +450,15 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     // dense once compaction would save less than a third of the ring: from there on
     // nearly every coordinate is selected and streaming beats per-coordinate work
     else if (dense_total <= 1.5L * compact_total &&
-             !(cfg->flags & (ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_PIPELINED_KERNEL))) {
+             !(cfg->flags & (ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_PIPELINED_KERNEL |
+                               ASYNCMESH_FLAG_OWNER_KERNEL))) {
         h->mode = kDense; h->n_slots = h->lag;
     }
     else { h->mode = kCompact; h->n_slots = h->lag + 1; }
 
     // the compact ring has two kernels; which one is fixed for the handle's life
-    h->pipelined = 0;   // 0 direct, 1 pipelined wide, 2 pipelined narrow, 3 pipelined narrow synchronous
+    h->pipelined = 0;   // 0 direct, 1 pipelined wide, 2 pipelined narrow, 3 pipelined narrow synchronous,
+                        // 4 to 6 owner (below)
     // synchronous mode: the stash route pays while most float4 groups are only partly
     // selected; towards p = 1 the direct kernel writes whole groups and wins
     if (h->mode == kSync && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
@@ -464,8 +470,23 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
             h->pipelined = 2;
     }
 
-    // E4M3 exchange and the eager estimate: the kernels' general form
-    const bool general = h->wire == 2u || h->correction == ASYNCMESH_CORRECTION_EAGER;
+    // Up to four replicas: the owner kernel (4: few ring / d entries fetched ahead per
+    // group, 5: many, 6: synchronous) wherever one of the two pipelined shapes would run,
+    // unless a flag asks for another kernel.  1B layout, tau = 4, ms per step, pipelined
+    // against owner: p = 0.01 21.6 / 20.7, 0.05 23.4 / 22.7, 0.1 26.2 / 23.9, 0.25 30.9 / 25.6,
+    // 0.5 37.4 / 29.0; tau = 0: 20.8 to 24.4 / 20.5 to 20.7 at every p.
+    const bool owner_asked = (cfg->flags & ASYNCMESH_FLAG_OWNER_KERNEL) != 0;
+    const bool owner_default =
+        !(cfg->flags & (ASYNCMESH_FLAG_DIRECT_KERNEL | ASYNCMESH_FLAG_PIPELINED_KERNEL)) &&
+        (h->mode == kCompact || (h->mode == kSync && cfg->p <= 0.8));
+    if (R <= 4 && h->mode != kDense && (owner_asked || owner_default)) {
+        const double mean = 128.0 * kOwnerV * cfg->p, sd = std::sqrt(mean * (1.0 - cfg->p));
+        h->pipelined = h->mode == kSync ? 6 : (mean + 4.0 * sd <= (double)kOwnerEntriesFew ? 4 : 5);
+    }
+
+    // E4M3 exchange, the eager estimate and NAdamW: the kernels' general form
+    const bool general = h->wire == 2u || h->correction == ASYNCMESH_CORRECTION_EAGER ||
+                         h->optimizer == ASYNCMESH_OPT_NADAMW;
 
     auto bail = [&](int code, const char *what) {
         release_all(h);
@@ -663,6 +684,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.wire = h->wire;
     P.eager = h->correction == ASYNCMESH_CORRECTION_EAGER ? 1u : 0u;
     P.nesterov = h->optimizer == ASYNCMESH_OPT_NADAMW ? 1u : 0u;
+    P.eps_inrange = (P.eps <= 1.152921504606847e18f) ? 1u : 0u;   // 2^60, see rounded_math.cuh
     double mu_product = h->mu_product;
     if (P.nesterov) {   // mu_t, mu_{t+1} and the running product of the momentum schedule
         const double mu_t = h->beta1 * (1.0 - 0.5 * std::pow(0.96, (double)t * h->momentum_decay));

@@ -4,6 +4,7 @@
 // side by side; this header is what the host code sees of them.
 #pragma once
 #include "step_kernel_pipelined.cuh"
+#include "step_kernel_owner.cuh"
 
 namespace amk {
 
@@ -26,5 +27,17 @@ KernelChoice pick_pipelined_few_common(uint32_t R, int shape, uint32_t S);     /
 KernelChoice pick_pipelined_few_general(uint32_t R, int shape, uint32_t S);
 KernelChoice pick_pipelined_many_common(uint32_t R, int shape, uint32_t S);    // R = 9..16
 KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S);
+// Owner kernel (R = 1..4).  mode: kCompact or kSync; entries: ring / d entries per group
+// of 256 coordinates fetched ahead (kOwnerEntriesFew or kOwnerEntriesMany).
+// Shape, measured on the 1B layout (R = 4, p = 0.05, ms per step): one replica row per
+// unit and 8 coordinates per lane (1 KB contiguous per array row and request) 22.7;
+// two rows per unit 23.0; 4 coordinates per lane (512-byte requests) 24.3 to 24.8 whatever
+// the rows per unit: the request size is worth 1 ms, also with nothing selected.
+constexpr int kOwnerStages = 3;
+constexpr int kOwnerV = 2;
+constexpr int kOwnerEntriesFew = 32, kOwnerEntriesMany = 128;
+constexpr int owner_ru(int) { return 1; }
+KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S);
+KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S);
 
 }  // namespace amk

@@ -40,6 +40,7 @@
 #include <cuda_runtime.h>
 
 #include "philox.cuh"
+#include "rounded_math.cuh"
 
 namespace amk {
 
@@ -86,7 +87,9 @@ struct StepParams {
     uint32_t wire;               // snapshots enter the average as fp32 (0), rounded to bfloat16 (1)
                                  // or to 8-bit floating point E4M3 (2)
     uint32_t eager;              // staleness estimate: 0 Eq. "ema", 1 d = (w^ - w^_old) / R
-    uint32_t nesterov;           // 0: AdamW, 1: NAdamW
+    uint32_t nesterov;           // 0: AdamW, 1: NAdamW (general form only)
+    uint32_t eps_inrange;        // eps is at most 2^60: sqrt(v^) + eps then stays in the range of the
+                                 // straight-line division whenever v^ is in the square root's
     float cg, cm;                // NAdamW: weights of the gradient and momentum parts
 };
 
@@ -132,26 +135,75 @@ __device__ __forceinline__ float staleness(const StepParams &P, float d, float d
     return __fadd_rn(__fmul_rn(P.oml, d), __fmul_rn(P.lam, diff));
 }
 
-// The local optimizer step (first line of Eq. "sparta"), one rounding per written
-// operation: AdamW with decoupled weight decay and bias correction, or NAdamW.
-__device__ __forceinline__ void adamw(const StepParams &P, float w, float g, float &m,
-                                      float &v, float &what)
+// u = m^ / (sqrt(v^) + eps) with the toolkit's correctly rounded routines: the route
+// of a coordinate group with an operand outside the range of the straight-line
+// forms (zero or subnormal moments, huge gradients, Inf, NaN).  Out of line, so that
+// the common route carries none of its code.
+static __device__ __noinline__ float adam_quotient_anyrange(float mh, float vh, float eps)
 {
-    m = __fadd_rn(__fmul_rn(P.b1, m), __fmul_rn(P.omb1, g));
-    v = __fadd_rn(__fmul_rn(P.b2, v), __fmul_rn(P.omb2, __fmul_rn(g, g)));
-    const float mh = __fmul_rn(m, P.ib1);
-    const float vh = __fmul_rn(v, P.ib2);
-    const float den = __fadd_rn(__fsqrt_rn(vh), P.eps);
-    const float decayed = __fsub_rn(w, __fmul_rn(P.lrwd, w));
-    if (P.nesterov == 0u) {
-        const float u = __fdiv_rn(mh, den);
-        what = __fsub_rn(decayed, __fmul_rn(P.lr, u));
+    return __fdiv_rn(mh, __fadd_rn(__fsqrt_rn(vh), eps));
+}
+
+// The local optimizer step (first line of Eq. "sparta") for NC coordinates of one
+// replica, one rounding per written operation: AdamW with decoupled weight decay and
+// bias correction; in the general form (GEN) also NAdamW.
+// AdamW's square root and division are the straight-line forms of rounded_math.cuh
+// when every operand of the group lies in their range (one test per group; eps is
+// tested by the host: P.eps_inrange), else the toolkit's routines: the same bits
+// either way.
+template <bool GEN, int NC>
+__device__ __forceinline__ void adamw_group(const StepParams &P, const float (&w)[NC],
+                                            const float (&g)[NC], float (&m)[NC], float (&v)[NC],
+                                            float (&what)[NC])
+{
+    float mh[NC], vh[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        m[c] = __fadd_rn(__fmul_rn(P.b1, m[c]), __fmul_rn(P.omb1, g[c]));
+        v[c] = __fadd_rn(__fmul_rn(P.b2, v[c]), __fmul_rn(P.omb2, __fmul_rn(g[c], g[c])));
+        mh[c] = __fmul_rn(m[c], P.ib1);
+        vh[c] = __fmul_rn(v[c], P.ib2);
+    }
+    if constexpr (GEN) {
+        if (P.nesterov != 0u) {
+            // NAdamW (Appendix B.1): gradient part and (uncorrected) momentum part over
+            // the same denominator, weighted by the momentum schedule's cg and cm
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const float den = __fadd_rn(__fsqrt_rn(vh[c]), P.eps);
+                const float decayed = __fsub_rn(w[c], __fmul_rn(P.lrwd, w[c]));
+                const float ug = __fdiv_rn(g[c], den);
+                const float um = __fdiv_rn(m[c], den);
+                what[c] = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug)), __fmul_rn(P.cm, um));
+            }
+            return;
+        }
+    }
+    float u[NC];
+    // (min / max drop a NaN operand: a NaN then takes the straight-line route and
+    // comes out as a NaN there too)
+    float vlo = vh[0], vhi = vh[0], alo = fabsf(mh[0]), ahi = fabsf(mh[0]);
+#pragma unroll
+    for (int c = 1; c < NC; ++c) {
+        vlo = fminf(vlo, vh[c]);
+        vhi = fmaxf(vhi, vh[c]);
+        alo = fminf(alo, fabsf(mh[c]));
+        ahi = fmaxf(ahi, fabsf(mh[c]));
+    }
+    const bool inrange = P.eps_inrange != 0u && vlo >= kSqrtLo && vhi <= kSqrtHi &&
+                         alo >= kDivNumLo && ahi <= kDivNumHi;
+    if (inrange) {
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
+            u[c] = div_rn_inrange(mh[c], __fadd_rn(sqrt_rn_inrange(vh[c]), P.eps));
     } else {
-        // NAdamW (Appendix B.1): gradient part and (uncorrected) momentum part over
-        // the same denominator, weighted by the momentum schedule's cg and cm
-        const float ug = __fdiv_rn(g, den);
-        const float um = __fdiv_rn(m, den);
-        what = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug)), __fmul_rn(P.cm, um));
+#pragma unroll
+        for (int c = 0; c < NC; ++c) u[c] = adam_quotient_anyrange(mh[c], vh[c], P.eps);
+    }
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const float decayed = __fsub_rn(w[c], __fmul_rn(P.lrwd, w[c]));
+        what[c] = __fsub_rn(decayed, __fmul_rn(P.lr, u[c]));
     }
 }
 
@@ -305,11 +357,9 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                     const float old[4] = {o4.x, o4.y, o4.z, o4.w};
                     float dd[4] = {d4[ii].x, d4[ii].y, d4[ii].z, d4[ii].w};
                     float wh[4], wn[4];
+                    adamw_group<GEN, 4>(P, w, g, m, v, wh);
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        adamw(P, w[c], g[c], m[c], v[c], wh[c]);
-                        wn[c] = wh[c];
-                    }
+                    for (int c = 0; c < 4; ++c) wn[c] = wh[c];
                     st_stream(st.M + off, m);
                     st_stream(st.V + off, v);
                     if (cm) {   // Eq. "ema" + corrected averaging on S^{t-tau}
@@ -410,11 +460,9 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                 float m[4] = {m4[ii].x, m4[ii].y, m4[ii].z, m4[ii].w};
                 float v[4] = {v4[ii].x, v4[ii].y, v4[ii].z, v4[ii].w};
                 float wh[4], wn[4];
+                adamw_group<GEN, 4>(P, w, g, m, v, wh);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    adamw(P, w[c], g[c], m[c], v[c], wh[c]);
-                    wn[c] = wh[c];
-                }
+                for (int c = 0; c < 4; ++c) wn[c] = wh[c];
                 st_stream(st.M + off, m);
                 st_stream(st.V + off, v);
 

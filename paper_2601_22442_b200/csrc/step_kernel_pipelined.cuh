@@ -420,24 +420,31 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                 wr = (wr + 1 == NST) ? 0 : wr + 1;
                 // (lanes past the end of the stage compute on whatever their slot
                 // holds: nothing of it is stored, stashed or selected)
-                float wn[V][4], wo[V][4];
+                float wn[V * 4], wo[V * 4];
+                {
+                    float g[V * 4], m[V * 4], v[V * 4];
 #pragma unroll
-                for (int h = 0; h < V; ++h) {
-                    const float4 w4 = *reinterpret_cast<const float4 *>(slot + (0 * V + h) * 512);
-                    const float4 g4 = *reinterpret_cast<const float4 *>(slot + (1 * V + h) * 512);
-                    const float4 m4 = *reinterpret_cast<const float4 *>(slot + (2 * V + h) * 512);
-                    const float4 v4 = *reinterpret_cast<const float4 *>(slot + (3 * V + h) * 512);
-                    const float g[4] = {g4.x, g4.y, g4.z, g4.w};
-                    float m[4] = {m4.x, m4.y, m4.z, m4.w};
-                    float v[4] = {v4.x, v4.y, v4.z, v4.w};
-                    wo[h][0] = w4.x; wo[h][1] = w4.y; wo[h][2] = w4.z; wo[h][3] = w4.w;
+                    for (int h = 0; h < V; ++h) {
+                        const float4 w4 = *reinterpret_cast<const float4 *>(slot + (0 * V + h) * 512);
+                        const float4 g4 = *reinterpret_cast<const float4 *>(slot + (1 * V + h) * 512);
+                        const float4 m4 = *reinterpret_cast<const float4 *>(slot + (2 * V + h) * 512);
+                        const float4 v4 = *reinterpret_cast<const float4 *>(slot + (3 * V + h) * 512);
+                        wo[4 * h] = w4.x; wo[4 * h + 1] = w4.y; wo[4 * h + 2] = w4.z; wo[4 * h + 3] = w4.w;
+                        g[4 * h] = g4.x; g[4 * h + 1] = g4.y; g[4 * h + 2] = g4.z; g[4 * h + 3] = g4.w;
+                        m[4 * h] = m4.x; m[4 * h + 1] = m4.y; m[4 * h + 2] = m4.z; m[4 * h + 3] = m4.w;
+                        v[4 * h] = v4.x; v[4 * h + 1] = v4.y; v[4 * h + 2] = v4.z; v[4 * h + 3] = v4.w;
+                    }
+                    adamw_group<GEN, V * 4>(P, wo, g, m, v, wn);
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) adamw(P, wo[h][c], g[c], m[c], v[c], wn[h][c]);
-                    const uint64_t mu = mu0 + (uint64_t)h * 128;
-                    if (mu < N) {
-                        const uint64_t off = (uint64_t)i * stride + mu;
-                        st_stream(st.M + off, m);
-                        st_stream(st.V + off, v);
+                    for (int h = 0; h < V; ++h) {
+                        const uint64_t mu = mu0 + (uint64_t)h * 128;
+                        if (mu < N) {
+                            const uint64_t off = (uint64_t)i * stride + mu;
+                            __stcs(reinterpret_cast<float4 *>(st.M + off),
+                                   make_float4(m[4 * h], m[4 * h + 1], m[4 * h + 2], m[4 * h + 3]));
+                            __stcs(reinterpret_cast<float4 *>(st.V + off),
+                                   make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]));
+                        }
                     }
                 }
 
@@ -446,8 +453,8 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     for (int j = 0; j < NB; ++j) {
                         if ((sm >> j) & 1u) {
                             const uint32_t r = uexcl + __popc(um & ((1u << j) - 1u));
-                            st_what[r * R + i] = wn[j >> 2][j & 3];
-                            st_wold[r * R + i] = wo[j >> 2][j & 3];
+                            st_what[r * R + i] = wn[j];
+                            st_wold[r * R + i] = wo[j];
                         }
                     }
                 }
@@ -456,7 +463,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                     for (int j = 0; j < NB; ++j) {
                         if ((om >> j) & 1u) {
                             const uint32_t below = (1u << j) - 1u;
-                            const float whj = wn[j >> 2][j & 3];
+                            const float whj = wn[j];
                             if ((cm >> j) & 1u) {
                                 const uint64_t ce = (uint64_t)(cfirst + __popc(cm & below)) * R;
                                 float old[R];
@@ -472,7 +479,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                                 const float diff = __fsub_rn(whj, old_i);
                                 const float dn = staleness<GEN>(P, *dp, diff);
                                 *dp = dn;
-                                wn[j >> 2][j & 3] = __fadd_rn(abar, dn);
+                                wn[j] = __fadd_rn(abar, dn);
                             }
                             if ((pm >> j) & 1u)
                                 ring_prod[(uint64_t)(pfirst + __popc(pm & below)) * R + i] = whj;
@@ -487,13 +494,14 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         const uint64_t off = (uint64_t)i * stride + mu;
                         // w and the look-ahead stay in L2 with normal priority: the few
                         // selected coordinates of these lines are patched a moment later
-                        st_keep(st.W + off, wn[h]);
+                        __stcg(reinterpret_cast<float4 *>(st.W + off),
+                               make_float4(wn[4 * h], wn[4 * h + 1], wn[4 * h + 2], wn[4 * h + 3]));
                         if (has_look) {   // Section 2.2: extrapolate the last update direction
                             float lk[4];
 #pragma unroll
                             for (int c = 0; c < 4; ++c)
-                                lk[c] = __fadd_rn(wn[h][c],
-                                                  __fmul_rn(delta, __fsub_rn(wn[h][c], wo[h][c])));
+                                lk[c] = __fadd_rn(wn[4 * h + c],
+                                                  __fmul_rn(delta, __fsub_rn(wn[4 * h + c], wo[4 * h + c])));
                             st_keep(st.LOOK + off, lk);
                         }
                     }

@@ -1,11 +1,12 @@
-// Instantiations of the step kernels.  Compiled seven times, -DAM_PART=0..6:
+// Instantiations of the step kernels.  Compiled nine times, -DAM_PART=0..8:
 // 0 direct kernel R = 1..8; 1 direct kernel R = 9..16, common form; 2 the same,
 // general form; 3 / 4 pipelined kernel R = 1..8, common / general form; 5 / 6
-// pipelined kernel R = 9..16, common / general form.
+// pipelined kernel R = 9..16, common / general form; 7 / 8 owner kernel R = 1..4,
+// common / general form.
 #include "kernel_table.cuh"
 
 #ifndef AM_PART
-#error "compile with -DAM_PART=0..6"
+#error "compile with -DAM_PART=0..8"
 #endif
 
 namespace amk {
@@ -65,6 +66,44 @@ KernelChoice pick_direct_many_general(uint32_t R, int mode)
     }
 }
 #endif
+
+#elif AM_PART >= 7   // owner kernel
+
+constexpr bool kGeneral = (AM_PART == 8);
+
+template <int R, int E, int MODE>
+static KernelChoice owner_as(uint32_t S)
+{
+    KernelChoice c;
+    c.fn = asyncmesh_step_kernel_owner<R, owner_ru(R), kOwnerV, kOwnerStages, E, MODE, kGeneral>;
+    c.threads = kOwnerThreads;
+    c.smem = (size_t)pipe_table_bytes(S) +
+             (size_t)(kOwnerThreads / 32) * OwnerCfg<R, owner_ru(R), kOwnerV, E>::warp_bytes(kOwnerStages);
+    return c;
+}
+
+template <int R>
+static KernelChoice owner(int mode, int entries, uint32_t S)
+{
+    if (mode == kSync) return owner_as<R, 1, kSync>(S);
+    return entries == kOwnerEntriesFew ? owner_as<R, kOwnerEntriesFew, kCompact>(S)
+                                       : owner_as<R, kOwnerEntriesMany, kCompact>(S);
+}
+
+#if AM_PART == 7
+KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S)
+#else
+KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S)
+#endif
+{
+    switch (R) {
+    case 1: return owner<1>(mode, entries, S);
+    case 2: return owner<2>(mode, entries, S);
+    case 3: return owner<3>(mode, entries, S);
+    case 4: return owner<4>(mode, entries, S);
+    default: return KernelChoice();
+    }
+}
 
 #else   // pipelined kernel
 

@@ -141,12 +141,18 @@ def test_modes_small(tau, p):
     run_case(4, [5000, 3 * 1024 + 17], p, tau, 0.9, steps=3 * tau + 4)
 
 
-@pytest.mark.parametrize("flag", ["direct", "pipelined"])
-@pytest.mark.parametrize("R,p", [(4, 0.05), (8, 0.3), (3, 0.7), (2, 1.0), (5, 0.0)])
-def test_both_synchronous_kernels(flag, R, p):
-    # tau = 0 (Eq. "sparta") through the direct kernel and through the stash route
+def kernel_flag(name):
     from paper_2601_22442_b200 import binding
-    f = binding.FLAG_DIRECT_KERNEL if flag == "direct" else binding.FLAG_PIPELINED_KERNEL
+    return {"direct": binding.FLAG_DIRECT_KERNEL, "pipelined": binding.FLAG_PIPELINED_KERNEL,
+            "owner": binding.FLAG_OWNER_KERNEL}[name]
+
+
+@pytest.mark.parametrize("flag", ["direct", "pipelined", "owner"])
+@pytest.mark.parametrize("R,p", [(4, 0.05), (8, 0.3), (3, 0.7), (2, 1.0), (5, 0.0), (1, 0.5)])
+def test_all_synchronous_kernels(flag, R, p):
+    # tau = 0 (Eq. "sparta") through the direct kernel, through the stash route and (up to
+    # four replicas; beyond, the flag changes nothing) in the owning lane's registers
+    f = kernel_flag(flag)
     run_case(R, [9000, 1024 * 3 + 5, 77], p, 0, 0.9, steps=5, flags=f)
     run_case(R, [5000], p, 0, 0.9, steps=6, flags=f, avg_interval=2, exchange="bf16")
 
@@ -158,14 +164,15 @@ def test_replica_counts(R):
     run_case(R, [2500], 0.3, 0, 0.9, steps=3)
 
 
-@pytest.mark.parametrize("flag", ["direct", "pipelined"])
-@pytest.mark.parametrize("R,p", [(4, 0.05), (8, 0.05), (3, 0.1), (4, 0.5), (8, 0.35), (2, 1.0), (5, 0.9)])
-def test_both_compact_ring_kernels(flag, R, p):
-    # the register-load kernel and the shared-memory pipelined kernel are two routes
-    # to the same numbers; large p forces the pipelined kernel through its in-place
-    # path (more selected coordinates per sub-iteration than its stash holds)
-    from paper_2601_22442_b200 import binding
-    f = binding.FLAG_DIRECT_KERNEL if flag == "direct" else binding.FLAG_PIPELINED_KERNEL
+@pytest.mark.parametrize("flag", ["direct", "pipelined", "owner"])
+@pytest.mark.parametrize("R,p", [(4, 0.05), (8, 0.05), (3, 0.1), (4, 0.5), (8, 0.35), (2, 1.0), (5, 0.9),
+                                 (1, 0.3), (4, 1.0)])
+def test_all_compact_ring_kernels(flag, R, p):
+    # the register-load kernel, the shared-memory pipelined kernel and the owner kernel are
+    # three routes to the same numbers; large p forces the pipelined kernel through its
+    # in-place path (more selected coordinates per sub-iteration than its stash holds) and
+    # the owner kernel past the ring / d entries it fetches ahead
+    f = kernel_flag(flag)
     run_case(R, [9000, 1024 * 3 + 5, 77], p, 2, 0.9, steps=7, flags=f)
 
 
@@ -184,6 +191,7 @@ def test_averaging_interval(K, tau, p):
     run_case(4, [5000, 1024 * 2 + 3], p, tau, 0.9, steps=4 * K + tau + 1, avg_interval=K)
     run_case(3, [5000], p, tau, 0.9, steps=3 * K + tau + 1, avg_interval=K,
              flags=binding.FLAG_DIRECT_KERNEL)
+    run_case(8, [5000], p, tau, 0.9, steps=3 * K + tau + 1, avg_interval=K)   # pipelined kernel
 
 
 @pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (2, 0.4)])
@@ -194,6 +202,7 @@ def test_nadamw(tau, p):
     run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp)
     run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
              flags=binding.FLAG_DIRECT_KERNEL)
+    run_case(6, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp)   # pipelined kernel
 
 
 @pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (3, 0.4)])
@@ -203,6 +212,8 @@ def test_bf16_exchange(tau, p):
     o, g = run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 5, exchange="bf16")
     run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="bf16",
              flags=binding.FLAG_DIRECT_KERNEL)
+    run_case(4, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="bf16",
+             flags=binding.FLAG_PIPELINED_KERNEL)
     # and it is not the fp32 exchange
     ref = oracle.Oracle(4, [6000, 1024 + 9], p=p, tau=tau, ema_beta=0.9, **HP)
     for s, n in enumerate([6000, 1024 + 9]):
@@ -219,6 +230,8 @@ def test_fp8_exchange(tau, p):
     o, g = run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 5, exchange="fp8")
     run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="fp8",
              flags=binding.FLAG_DIRECT_KERNEL)
+    run_case(4, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="fp8",
+             flags=binding.FLAG_PIPELINED_KERNEL)
     ref = oracle.Oracle(4, [6000, 1024 + 9], p=p, tau=tau, ema_beta=0.9, exchange="bf16", **HP)
     for s, n in enumerate([6000, 1024 + 9]):
         ref.init_params(s, si.init_weights_host(0x1217, s, 0, n))
@@ -268,6 +281,8 @@ def test_eager_staleness_estimate(p, tau, K):
         assert np.abs(g.get(0, "d")).max() > 0
     run_case(3, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
              flags=binding.FLAG_DIRECT_KERNEL)
+    run_case(4, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
+             flags=binding.FLAG_PIPELINED_KERNEL)
     if 0 < p < 1 and tau:
         run_case(3, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
                  flags=binding.FLAG_DENSE_RING)
