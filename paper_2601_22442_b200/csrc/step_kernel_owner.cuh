@@ -403,16 +403,29 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                     uint32_t e[NB];
                     const uint32_t total = owner_ranks<NB>(pm, lt, e);
                     if (pm) {
+                        // A scattered store instruction costs the memory pipeline about the same
+                        // with one lane taking part as with all of them, and most lanes have at
+                        // most one entry per group: a lane holds its first entry back, so that one
+                        // store instruction at the end serves the first entries of all lanes.
                         float *ring_at = ring_prod + (uint64_t)(pbase + prun) * R;
+                        float held[R];
+                        uint32_t held_e = kInvalidBase;
 #pragma unroll
                         for (int j = 0; j < NB; ++j) {
                             if ((pm >> j) & 1u) {
                                 float x[R];
 #pragma unroll
                                 for (int i = 0; i < R; ++i) x[i] = wn[i][j];
-                                store_replicas<R>(ring_at + (uint64_t)e[j] * R, x);
+                                if (held_e == kInvalidBase) {
+                                    held_e = e[j];
+#pragma unroll
+                                    for (int i = 0; i < R; ++i) held[i] = x[i];
+                                } else {
+                                    store_replicas<R>(ring_at + (uint64_t)e[j] * R, x);
+                                }
                             }
                         }
+                        store_replicas<R>(ring_at + (uint64_t)held_e * R, held);
                     }
                     prun += total;
                 }
@@ -436,6 +449,8 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                             }
                         };
                         if constexpr (Cfg::kPair) {
+                            float held_d[8];
+                            float *held_dp = nullptr;
 #pragma unroll
                             for (int q = 0; q < NB / 2; ++q) {   // pairs of coordinates = sectors of d
                                 const uint32_t pc = (cm >> (2 * q)) & 3u;
@@ -460,9 +475,16 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                                             for (int i = 0; i < R; ++i) dpair[R * c + i] = dd[i];
                                         }
                                     }
-                                    st_sector(dp, dpair);
+                                    if (held_dp == nullptr) {   // held back, as for the ring entries above
+                                        held_dp = dp;
+#pragma unroll
+                                        for (int x = 0; x < 8; ++x) held_d[x] = dpair[x];
+                                    } else {
+                                        st_sector(dp, dpair);
+                                    }
                                 }
                             }
+                            st_sector(held_dp, held_d);
                         } else {
 #pragma unroll
                             for (int j = 0; j < NB; ++j) {
