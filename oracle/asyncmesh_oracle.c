@@ -226,7 +226,8 @@ int am_oracle_init_params(am_oracle *o, uint32_t stage, int32_t replica,
 
 /*
  * What a replica's snapshot value looks like to the others.  The paper's
- * quantisation study (Section 4 "robustness", Appendix B.2) sends the subset in
+ * quantisation study (Section 5.3, paragraph "Robustness of Sparse Averaging";
+ * Appendix B.2) sends the subset in
  * reduced precision; with exchange = 1 every value entering the average is
  * first rounded to bfloat16 (round to nearest even: keep the upper 16 bits of
  * the binary32 pattern), with exchange = 2 to 8-bit floating point (E4M3, the
@@ -393,11 +394,14 @@ int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
             }
         }
 
-        /* O4: look-ahead by the stage's delay */
+        /* O4: look-ahead by the stage's delay.  With delay 0 nothing is
+         * extrapolated: the look-ahead weights ARE the current weights (the
+         * product w + 0 * (w - w_prev) is not that for w = +-Inf, where it is
+         * NaN, nor for w = -0, where it is +0). */
         const float delta = (float)o->delay[s];
         for (uint64_t k = 0; k < (uint64_t)R * N; ++k) {
             const float dir = w[k] - wprev[k];
-            look[k] = w[k] + (delta * dir);
+            look[k] = o->delay[s] == 0 ? w[k] : w[k] + (delta * dir);
         }
     }
     return 0;
@@ -436,7 +440,7 @@ int am_oracle_lookahead(const am_oracle *o, uint32_t stage, uint32_t delay, floa
     const float delta = (float)delay;
     for (uint64_t k = 0; k < n; ++k) {
         const float dir = o->w[stage][k] - o->wprev[stage][k];
-        dst[k] = o->w[stage][k] + (delta * dir);
+        dst[k] = delay == 0 ? o->w[stage][k] : o->w[stage][k] + (delta * dir);   /* delay 0: w itself */
     }
     return 0;
 }

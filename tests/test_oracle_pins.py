@@ -306,6 +306,27 @@ def test_lookahead_zero_delay_is_identity():
         assert (o.get(1, "look") == o.get(1, "w")).all()
 
 
+def test_lookahead_zero_delay_is_identity_on_infinite_and_signed_zero_weights():
+    # "the look-ahead with zero delay returns the current weights": bit for bit, also where
+    # w + 0 * (w - w_prev) would not (0 * (Inf - Inf) is NaN; -0 + 0 is +0)
+    w0 = np.array([np.inf, -np.inf, -0.0, 0.0, 3e38, -3e38, 1.0, np.nan], dtype=np.float32)
+    hp = dict(HP, weight_decay=0.0)
+    o = oracle.Oracle(1, [w0.size, w0.size], p=0.0, tau=1, ema_beta=0.9, lookahead_delay=[0, 2], **hp)
+    o.init_params(0, w0); o.init_params(1, w0)
+    g = np.zeros((1, w0.size), dtype=np.float32)
+    for _ in range(3):
+        o.step([g, g])
+        w, look = o.get(0, "w"), o.get(0, "look")
+        assert np.array_equal(w.view(np.uint32), look.view(np.uint32))
+        assert np.array_equal(o.lookahead(0, 0).view(np.uint32), w.view(np.uint32))
+        assert np.array_equal(o.lookahead(1, 0).view(np.uint32), o.get(1, "w").view(np.uint32))
+    # before any step w^{-1} = w^0: with a delay the formula applies, and Inf - Inf is NaN
+    o3 = oracle.Oracle(1, [w0.size], p=0.0, tau=1, ema_beta=0.9, lookahead_delay=[2], **hp)
+    o3.init_params(0, w0)
+    assert np.isnan(o3.lookahead(0, 2)[0, 0]) and o3.lookahead(0, 0)[0, 0] == np.inf
+    assert np.signbit(o3.lookahead(0, 0)[0, 2]) and not np.signbit(o3.lookahead(0, 2)[0, 2])
+
+
 def test_lookahead_default_delay_and_constant_velocity():
     # default delay is S-1-stage; with a constant update direction the
     # extrapolation by k steps lands on the weights k steps later
