@@ -108,6 +108,125 @@ def test_config_llama1b_20_steps():
     run_full(w["R"], w["numel"], 0.05, w["tau"], w["steps"])
 
 
+def test_config_llama125m_whole_state():
+    """Every coordinate of every replica of the 125M configuration after its 50 steps, not
+    slices: the oracle replays the stages in ranges of 2^20 coordinates on all host cores
+    (child processes), the ranges' digests are compared with digests of the same ranges
+    read back from the library."""
+    import multiprocessing as mp
+    import os
+    import paper_2601_22442_b200 as pkg
+    from paper_2601_22442_b200.layouts import DEFAULT_HP
+    from tests import whole_state_worker as wk
+    w = workloads()["llama125m"]
+    R, numel, tau, steps = w["R"], w["numel"], w["tau"], w["steps"]
+    p, lam, mesh_seed = DEFAULT_HP["p"], DEFAULT_HP["ema_beta"], 0x5EED
+    hp = {k: v for k, v in DEFAULT_HP.items() if k not in ("p", "ema_beta")}
+    chunk = 1 << 20
+    tasks = [(R, s, len(numel), b, min(chunk, n - b), p, tau, lam, hp, steps, GRAD_SEED, INIT_SEED, mesh_seed)
+             for s, n in enumerate(numel) for b in range(0, n, chunk)]
+    tasks.sort(key=lambda t: -t[4])
+    ctx = mp.get_context("spawn")
+    pool = ctx.Pool(max(1, min(os.cpu_count() or 1, 32)))
+    pending = pool.map_async(wk.replay, tasks, chunksize=1)
+
+    g = pkg.AsyncMesh(R, numel, tau=tau, seed=mesh_seed, **DEFAULT_HP)
+    dev = torch.device("cuda", 0)
+    for s, n in enumerate(numel):
+        tmp = torch.empty(n, dtype=torch.float32, device=dev)
+        si.normal_device(tmp, si.stream_key(INIT_SEED, si.KIND_INIT, 0, s, 0), 0, 0.02)
+        g.init_params(s, tmp)
+        del tmp
+    bufs = g.empty_grads()
+    for t in range(1, steps + 1):
+        for s, n in enumerate(numel):
+            si.grads_device(bufs[s], GRAD_SEED, t, s, n)
+        g.step(bufs)
+    g.status()
+    mine = {}
+    for task in tasks:
+        s, b, c = task[1], task[3], task[4]
+        mine[(s, b)] = {name: wk.digest(g.get_range(s, name, b, c)) for name in STATE_NAMES}
+    results = pending.get(timeout=3000)
+    pool.close()
+    pool.join()
+    assert len(results) == len(tasks)
+    covered = [0] * len(numel)
+    for s, b, c, dig in results:
+        covered[s] += c
+        for name in STATE_NAMES:
+            assert dig[name] == mine[(s, b)][name], (s, b, c, name)
+    assert covered == list(numel)
+    g.destroy()
+    del bufs
+    torch.cuda.empty_cache()
+
+
+def state_digests(flags, steps):
+    """Runs the 1B configuration with the kernel `flags` selects and returns, per stage and
+    state array, a digest computed on the device from the library's own buffers (found
+    through the allocator callbacks: the state arrays are the blocks of R x stride floats,
+    allocated in a fixed order)."""
+    import paper_2601_22442_b200 as pkg
+    from paper_2601_22442_b200.binding import TorchAllocator
+    from paper_2601_22442_b200.layouts import DEFAULT_HP
+    w = workloads()["llama1b"]
+    R, numel, tau = w["R"], w["numel"], w["tau"]
+
+    class Recording(TorchAllocator):
+        def __init__(self, dev):
+            super().__init__(dev)
+            self.order = []
+
+        def _alloc(self, ctx, nbytes):
+            ptr = super()._alloc(ctx, nbytes)
+            if ptr is not None:
+                self.order.append((ptr, int(nbytes)))
+            return ptr
+
+    alloc = Recording(0)
+    g = pkg.AsyncMesh(R, numel, tau=tau, flags=flags, allocator=alloc, **DEFAULT_HP)
+    dev = torch.device("cuda", 0)
+    for s, n in enumerate(numel):
+        tmp = torch.empty(n, dtype=torch.float32, device=dev)
+        si.normal_device(tmp, si.stream_key(INIT_SEED, si.KIND_INIT, 0, s, 0), 0, 0.02)
+        g.init_params(s, tmp)
+        del tmp
+    bufs = g.empty_grads()
+    for t in range(1, steps + 1):
+        for s, n in enumerate(numel):
+            si.grads_device(bufs[s], GRAD_SEED, t, s, n)
+        g.step(bufs)
+    g.status()
+    torch.cuda.synchronize()
+    sizes = {R * g.stride[s] * 4 for s in range(len(numel))}
+    out = []
+    for ptr, nbytes in alloc.order:
+        if nbytes in sizes and ptr in alloc._live:
+            x = alloc._live[ptr].view(torch.int32)
+            k = torch.arange(1, x.numel() + 1, dtype=torch.int64, device=dev)
+            out.append((nbytes, int(x.sum(dtype=torch.int64).item()), int((x.to(torch.int64) * k).sum().item())))
+            del k
+    g.destroy()
+    del bufs, alloc
+    torch.cuda.empty_cache()
+    return out
+
+
+def test_config_llama1b_three_kernels_leave_the_same_state():
+    """The whole state of the 1B configuration (every w, m, v, d and look-ahead value) after
+    8 steps is the same, bit for bit, through the owner kernel (the default there), the
+    pipelined kernel and the direct kernel.  A comparison of the library with itself: it
+    widens the coverage of the slice-based oracle comparison above, it does not replace it."""
+    from paper_2601_22442_b200 import binding
+    a = state_digests(0, 8)
+    assert len(a) == 8 * 4 + 7            # w, m, v, d per stage, look-ahead where the delay is not 0
+    b = state_digests(binding.FLAG_PIPELINED_KERNEL, 8)
+    assert a == b
+    c = state_digests(binding.FLAG_DIRECT_KERNEL, 8)
+    assert a == c
+
+
 @pytest.mark.parametrize("tau", [0, 1, 4, 8])
 @pytest.mark.parametrize("p", [0.01, 0.05, 0.25, 1.0])
 def test_config_sweep_on_350m_layout(p, tau):
