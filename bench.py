@@ -29,13 +29,25 @@ METRIC = "replica_param_updates_per_sec"
 UNIT = "replica*param/s"
 GRAD_SEED, INIT_SEED, MESH_SEED = 0x6AD5, 0x1217, 0x5EED
 
-# Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one
-# steady-state launch relative to its algorithmic bytes, from the ncu capture on
-# the small `profile` workload summarised under profiles/ (the full workloads are
-# too large to capture with many passes).  The kernel is a streaming scan, so
-# traffic grows with the units processed; the ratio scales it to any workload
-# that runs the same kernel (compact ring, p = 0.05, R = 4).
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"llama1b": 1.039, "profile": 1.039}
+def measured_traffic_ratio(kernel_name: str, p: float):
+    """DRAM traffic of one steady-state launch relative to its algorithmic bytes, as
+    measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) for the kernel the
+    handle actually runs, from the table kept next to the profile summaries
+    (profiles/dram_traffic.txt: kernel name | p | ratio | capture).  The captures are
+    taken on the small `profile` workload; the kernels are streaming scans whose traffic
+    grows with the units processed, so the ratio carries over to any workload that runs
+    the same kernel at the same p.  None when the table has no such entry."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    try:
+        for line in open(path):
+            if line.startswith("#") or "|" not in line:
+                continue
+            f = [x.strip() for x in line.split("|")]
+            if f[0] == kernel_name and abs(float(f[1]) - p) <= 1e-9:
+                return float(f[2])
+    except (OSError, ValueError, IndexError):
+        pass
+    return None
 
 
 def parse_args():
@@ -50,6 +62,8 @@ def parse_args():
     ap.add_argument("--tau", type=int, default=None)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--time-diagnostics", action="store_true",
+                    help="also time the consensus-error and EMA-spread reductions (CUDA events)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--flags", type=int, default=0, help="asyncmesh_config.flags (diagnostic)")
     ap.add_argument("--optimizer", choices=["adamw", "nadamw"], default="adamw",
@@ -293,6 +307,26 @@ def run_native(args):
     ms, units = aggregate_over_ranks(local_ms, units_per_step, world, dev)
     value = units / (ms * 1e-3)
 
+    kernel_name = mesh.kernel_name()
+    diagnostics = None
+    if args.time_diagnostics:
+        # the two read-only reductions, every stage, device time only
+        diagnostics = {}
+        for what, fn, per_rc in (("consensus_error", mesh.consensus_error, 4.0),
+                                 ("ema_variance", mesh.ema_variance, 4.0)):
+            for s in range(len(numel)):
+                fn(s)                                   # warm-up
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for s in range(len(numel)):
+                fn(s)
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            d_ms = e0.elapsed_time(e1)
+            gbs = per_rc * units_per_step / (d_ms * 1e-3) / 1e9
+            diagnostics[what] = {"ms_all_stages": d_ms, "read_GBs": gbs,
+                                 "frac_of_copy_peak": gbs / measured_peak_gbs()[0]}
+
     # ---- end to end: host gradients in, result out, every step ---------------
     e2e = None
     if not args.no_e2e:
@@ -331,9 +365,7 @@ def run_native(args):
 
     peak, peak_kind = measured_peak_gbs()
     achieved = min_bytes / (local_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_OVER_ALGORITHMIC.get(args.workload)
-    if args.p is not None or args.tau is not None:
-        traffic = None
+    traffic = measured_traffic_ratio(kernel_name, hp["p"])
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -342,12 +374,14 @@ def run_native(args):
                 "across timed steps, generated outside the timed region)",
         "config": config_dict(args, w, hp),
         "step_ms": {"min": min(per_step), "median": statistics.median(per_step), "max": max(per_step)},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "kernel": kernel_name,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
                      "frac_of_8TBs": achieved / 8000.0, "min_bytes_per_step": min_bytes,
                      "traffic": None if traffic is None else traffic * min_bytes},
     }
+    if diagnostics is not None:
+        line["diagnostics"] = diagnostics
     if world == 1 and not args.no_cpu_baseline:
         r = time_oracle(w, hp, steps=8, warmup=tau + 1, sample_per_stage=1 << 19)
         line["cpu_baseline"] = {"value": r["value"], "unit": UNIT, "cores": 1, "kind": "oracle",

@@ -65,8 +65,10 @@ extern "C" {
 #define ASYNCMESH_FLAG_PIPELINED_KERNEL 4u /* use the compact ring and the pipelined kernel for
                                              any p (diagnostic: exercises its in-place path) */
 #define ASYNCMESH_FLAG_OWNER_KERNEL 256u /* use the kernel in which the lane that owns a coordinate
-                                           does all of its work (up to four replicas, compact ring
-                                           or tau = 0) */
+                                           does all of its work, with the compact ring whatever p
+                                           is (up to four replicas; it is the default there for
+                                           the compact ring and for tau = 0, this flag only extends
+                                           it to subsets the dense ring would otherwise serve)  */
 #define ASYNCMESH_FLAG_BF16_EXCHANGE 16u /* the subset is exchanged in bfloat16 (the paper's
                                            quantisation study): every snapshot value entering the
                                            replica average is first rounded to bfloat16 (nearest
@@ -170,7 +172,8 @@ int asyncmesh_init_params(asyncmesh *h, uint32_t stage, int32_t replica,
                           const float *src, uint64_t n, int src_on_device);
 
 /* Floats between consecutive replica rows of a stage (a multiple of 32,
- * >= stage_numel[stage]).  Gradient buffers use the same stride. */
+ * >= stage_numel[stage]).  Gradient buffers use the same stride.  (Layout
+ * bookkeeping: defines nothing of the paper's method.) */
 int asyncmesh_row_stride(const asyncmesh *h, uint32_t stage, uint64_t *stride);
 
 /*
@@ -196,6 +199,8 @@ int asyncmesh_step_ex(asyncmesh *h, const float *const *grads,
  * asynchronous; pageable memory works and is slower.
  */
 int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host);
+int asyncmesh_step_host_ex(asyncmesh *h, const float *const *grads_host,
+                           double ema_beta_t, double lr_t);   /* per-step scalars as in asyncmesh_step_ex */
 
 /*
  * Look-ahead weights of a stage: w^t + delay * (w^t - w^{t-1}) (Section 2.2).
@@ -211,9 +216,9 @@ int asyncmesh_lookahead_weights(asyncmesh *h, uint32_t stage, uint32_t delay,
                                 const float **out_device, uint64_t *row_stride);
 
 /*
- * Copy out the weights of one replica (replica = -1: the replica mean, the
- * consensus model the paper evaluates, summed in replica order and divided by
- * R).  dst receives n = stage_numel[stage] floats, on the device if
+ * Copy out the weights of one replica (replica = -1: the replica mean, summed
+ * in replica order and divided by R -- the model the paper evaluates: Section 5.1
+ * reports validation loss on the average of the replicas' weights).  dst receives n = stage_numel[stage] floats, on the device if
  * dst_on_device != 0 else on the host.  Waits for the stream; reports a pending
  * device status (ring overflow) as DEVICE_STATUS.
  */
@@ -246,19 +251,9 @@ int asyncmesh_subset_mask(asyncmesh *h, uint32_t stage, uint64_t step,
 int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *out_host);
 
 /*
- * Spread of the staleness estimates across replicas (the appendix figure on the
- * consensus error plots the "variance between EMA estimates in each replica",
- * mean and max across the model dimension): per coordinate the population
- * variance (1/R) sum_i (d_i - dbar)^2, formed in double on the device;
- * *mean_host = its mean over the stage's coordinates, *max_host = its maximum
- * (host doubles, both required).  Waits for the stream.
- */
-int asyncmesh_ema_variance(asyncmesh *h, uint32_t stage, double *mean_host, double *max_host);
-
-/*
- * The same quantity for callers that cannot let the library allocate (the paper
- * has no counterpart: this is a packaging variant of the call above, not part
- * of the method).  Meant for hosts whose GPU memory is entirely owned by their
+ * The consensus error again (the quantity asyncmesh_consensus_error returns), for
+ * callers that cannot let the library allocate (the paper has no counterpart: this
+ * is a packaging variant of that call, not part of the method).  Meant for hosts whose GPU memory is entirely owned by their
  * own pool, for loops that must not hit the device-wide synchronisation an
  * allocation may cause, and for hooks that run where the process may not grow:
  * it calls no cudaMalloc / cudaFree and no allocating library routine.  The
@@ -272,8 +267,9 @@ int asyncmesh_ema_variance(asyncmesh *h, uint32_t stage, double *mean_host, doub
  *               split the rows and add the partial results
  *   out_host    host, receives sum_i ||w_i - wbar||^2 over the n coordinates
  *   device, stream   where to run; the call waits for the stream before returning
- * The first call on a device also looks up the scratch array's device address;
- * make that first call before any stream capture.  All calls share the one
+ * The first call on a device also looks up the scratch array's device address
+ * (with lazy module loading that is also when the array comes into existence on
+ * that device); make that first call before any stream capture.  All calls share the one
  * array and it keeps the last call's contents (every slot a call reads it has
  * written first, so nothing needs clearing); two calls whose kernels overlap on
  * the GPU (different streams, different threads) race on it and must be
@@ -283,14 +279,36 @@ int asyncmesh_consensus_error_noalloc(int device, void *stream, const float *w_d
                                       uint32_t R, uint64_t n, uint64_t row_stride,
                                       double *out_host);
 
-/* Steps taken so far. */
+/*
+ * Spread of the staleness estimates across replicas (the appendix figure on the
+ * consensus error plots the "variance between EMA estimates in each replica",
+ * mean and max across the model dimension): per coordinate the population
+ * variance (1/R) sum_i (d_i - dbar)^2, formed in double on the device;
+ * *mean_host = its mean over the stage's coordinates, *max_host = its maximum
+ * (host doubles, both required).  Waits for the stream.
+ */
+int asyncmesh_ema_variance(asyncmesh *h, uint32_t stage, double *mean_host, double *max_host);
+
+/* Steps taken so far.  (Bookkeeping, like asyncmesh_status and
+ * asyncmesh_last_error: defines nothing of the paper's method.) */
 int asyncmesh_step_count(const asyncmesh *h, uint64_t *t);
+
+/*
+ * Which step kernel the handle runs, as text, e.g.
+ * "owner R=4 compact entries=32": the kernel family (direct, pipelined, owner),
+ * the replica count it is compiled for, the ring mode (sync, compact, dense) and
+ * the shape parameter of the family.  Fixed at create.  Copies at most cap bytes
+ * including the terminating 0 into buf (host).  Measurements (DRAM traffic per
+ * launch, for instance) are filed under this name.  Bookkeeping only.
+ */
+int asyncmesh_kernel_name(const asyncmesh *h, char *buf, size_t cap);
 
 /*
  * Bytes the last step had to move at least: per replica-coordinate 16 read
  * (w, g, m, v) + 12 written (w, m, v), + 4 where the look-ahead is a separate
  * buffer, + 4p for the snapshot write, + 12p once averages are being consumed
  * (ring read, d read, d write).  Used as the numerator of the HBM roofline.
+ * (Bookkeeping: defines nothing of the paper's method.)
  */
 int asyncmesh_min_bytes_last_step(const asyncmesh *h, uint64_t *bytes);
 

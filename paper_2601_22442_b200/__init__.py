@@ -5,7 +5,8 @@ behind a C ABI (``include/asyncmesh.h``).  This package is the thin Python
 binding of that library plus the workload layouts."""
 from .binding import (AsyncMesh, AsyncMeshError, TorchAllocator, asyncmesh_create,  # noqa: F401
                       asyncmesh_destroy, asyncmesh_init_params, asyncmesh_step,
-                      asyncmesh_step_ex, asyncmesh_step_host, asyncmesh_lookahead_weights,
+                      asyncmesh_step_ex, asyncmesh_step_host, asyncmesh_step_host_ex,
+                      asyncmesh_kernel_name, asyncmesh_lookahead_weights,
                       asyncmesh_read_params, asyncmesh_read_state, asyncmesh_read_state_range,
                       asyncmesh_subset_mask,
                       asyncmesh_consensus_error, asyncmesh_consensus_error_noalloc,

@@ -72,6 +72,8 @@ SIGNATURES = {
     "asyncmesh_step": (_int, [_vp, ctypes.POINTER(_vp)]),
     "asyncmesh_step_ex": (_int, [_vp, ctypes.POINTER(_vp), ctypes.c_double, ctypes.c_double]),
     "asyncmesh_step_host": (_int, [_vp, ctypes.POINTER(_vp)]),
+    "asyncmesh_step_host_ex": (_int, [_vp, ctypes.POINTER(_vp), ctypes.c_double, ctypes.c_double]),
+    "asyncmesh_kernel_name": (_int, [_vp, ctypes.c_char_p, ctypes.c_size_t]),
     "asyncmesh_lookahead_weights": (_int, [_vp, _u32, _u32, ctypes.POINTER(_vp),
                                            ctypes.POINTER(_u64)]),
     "asyncmesh_read_params": (_int, [_vp, _u32, _i32, _vp, _u64, _int]),
@@ -259,7 +261,7 @@ class AsyncMesh:
         else:
             _check(load().asyncmesh_step_ex(self._h, ptrs, float(ema_beta_t), float(lr_t)))
 
-    def step_host(self, grads_host) -> None:
+    def step_host(self, grads_host, ema_beta_t: float = -1.0, lr_t: float = -1.0) -> None:
         """grads_host[j]: host float32 [R, numel_j], contiguous (numpy array or
         pinned CPU torch tensor)."""
         ptrs = []
@@ -271,7 +273,11 @@ class AsyncMesh:
             else:
                 assert (not g.is_cuda) and g.is_contiguous() and g.numel() == self.R * self.numel[j]
                 ptrs.append(g.data_ptr())
-        _check(load().asyncmesh_step_host(self._h, (_vp * self.S)(*ptrs)))
+        if ema_beta_t < 0 and lr_t < 0:
+            _check(load().asyncmesh_step_host(self._h, (_vp * self.S)(*ptrs)))
+        else:
+            _check(load().asyncmesh_step_host_ex(self._h, (_vp * self.S)(*ptrs), float(ema_beta_t),
+                                                 float(lr_t)))
 
     # -- results out ---------------------------------------------------------------
     def lookahead_weights(self, stage: int, delay: int):
@@ -344,6 +350,11 @@ class AsyncMesh:
     def status(self) -> None:
         _check(load().asyncmesh_status(self._h))
 
+    def kernel_name(self) -> str:
+        buf = ctypes.create_string_buffer(128)
+        _check(load().asyncmesh_kernel_name(self._h, buf, 128))
+        return buf.value.decode()
+
 
 # ---- the C names, as functions ---------------------------------------------------
 
@@ -371,6 +382,14 @@ def asyncmesh_step_ex(h: AsyncMesh, grads, ema_beta_t, lr_t) -> None:
 
 def asyncmesh_step_host(h: AsyncMesh, grads_host) -> None:
     h.step_host(grads_host)
+
+
+def asyncmesh_step_host_ex(h: AsyncMesh, grads_host, ema_beta_t, lr_t) -> None:
+    h.step_host(grads_host, ema_beta_t, lr_t)
+
+
+def asyncmesh_kernel_name(h: AsyncMesh) -> str:
+    return h.kernel_name()
 
 
 def asyncmesh_lookahead_weights(h: AsyncMesh, stage, delay):

@@ -96,6 +96,7 @@ struct asyncmesh {
 
     int mode = kSync;
     int pipelined = 0;
+    bool general = false;             // the kernels' general form (E4M3 exchange, eager estimate, NAdamW)
     KernelChoice kernel;
     uint32_t n_slots = 0;
     uint32_t total_chunks = 0;
@@ -176,21 +177,9 @@ __global__ void mean_rows_kernel(const float *W, uint32_t R, uint64_t stride, ui
     }
 }
 
-// sum over coordinates and replicas of (w_i - mean)^2, in double.
-__global__ void consensus_kernel(const float *W, uint32_t R, uint64_t stride, uint64_t N,
-                                 double *out)
+// Block-wide sum of a double into *out (one atomicAdd per block).
+__device__ __forceinline__ void block_sum_to(double acc, double *out)
 {
-    double acc = 0.0;
-    for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
-         mu += (uint64_t)gridDim.x * blockDim.x) {
-        double mean = 0.0;
-        for (uint32_t i = 0; i < R; ++i) mean += (double)W[(uint64_t)i * stride + mu];
-        mean /= (double)R;
-        for (uint32_t i = 0; i < R; ++i) {
-            const double e = (double)W[(uint64_t)i * stride + mu] - mean;
-            acc += e * e;
-        }
-    }
     for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
     __shared__ double part[32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -200,6 +189,54 @@ __global__ void consensus_kernel(const float *W, uint32_t R, uint64_t stride, ui
         acc = lane < (int)(blockDim.x >> 5) ? part[lane] : 0.0;
         for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
         if (lane == 0) atomicAdd(out, acc);
+    }
+}
+
+// sum over coordinates and replicas of (w_i - mean)^2, in double.  A thread takes four
+// consecutive coordinates (one 16-byte load per replica row; rows are padded to 32
+// floats and 16-byte aligned) and keeps the R x 4 values in registers between the two
+// passes, so every byte is read once: a read-only stream.
+template <int R>
+__global__ void consensus_kernel(const float *W, uint64_t stride, uint64_t N, double *out)
+{
+    double acc = 0.0;
+    const uint64_t n4 = (N + 3) / 4;
+    for (uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n4;
+         q += (uint64_t)gridDim.x * blockDim.x) {
+        float4 x[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) x[i] = __ldcs(reinterpret_cast<const float4 *>(W + (uint64_t)i * stride) + q);
+        const uint64_t left = N - 4 * q;   // coordinates of this group that exist (1..4 at the tail)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if ((uint64_t)c < left) {
+                double mean = 0.0;
+#pragma unroll
+                for (int i = 0; i < R; ++i) mean += (double)reinterpret_cast<const float *>(&x[i])[c];
+                mean /= (double)R;
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    const double e = (double)reinterpret_cast<const float *>(&x[i])[c] - mean;
+                    acc += e * e;
+                }
+            }
+        }
+    }
+    block_sum_to(acc, out);
+}
+
+typedef void (*consensus_fn)(const float *, uint64_t, uint64_t, double *);
+static consensus_fn consensus_for(uint32_t R)
+{
+    switch (R) {
+    case 1: return consensus_kernel<1>;   case 2: return consensus_kernel<2>;
+    case 3: return consensus_kernel<3>;   case 4: return consensus_kernel<4>;
+    case 5: return consensus_kernel<5>;   case 6: return consensus_kernel<6>;
+    case 7: return consensus_kernel<7>;   case 8: return consensus_kernel<8>;
+    case 9: return consensus_kernel<9>;   case 10: return consensus_kernel<10>;
+    case 11: return consensus_kernel<11>; case 12: return consensus_kernel<12>;
+    case 13: return consensus_kernel<13>; case 14: return consensus_kernel<14>;
+    case 15: return consensus_kernel<15>; default: return consensus_kernel<16>;
     }
 }
 
@@ -223,24 +260,54 @@ __global__ void extrapolate_kernel(const float *W, const float *Wprev, float *ou
 // Per coordinate the population variance of d over the replicas, in double;
 // out[0] accumulates the sum over coordinates, out[1] the maximum (variances are
 // non-negative, so their bit patterns order like unsigned integers).
-__global__ void spread_kernel(const float *D, uint32_t R, uint64_t coord_step, uint64_t replica_step,
-                              uint64_t N, double *out)
+// MAJOR 0: d is coordinate-major [stride][R], a thread takes one coordinate's R
+// contiguous floats (vector loads); MAJOR 1: replica-major [R][stride] (dense ring),
+// a thread takes four consecutive coordinates, one 16-byte load per row.  Either way
+// every byte is read once: a read-only stream.
+template <int R, int MAJOR>
+__global__ void spread_kernel(const float *D, uint64_t stride, uint64_t N, double *out)
 {
     double acc = 0.0, mx = 0.0;
-    for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
-         mu += (uint64_t)gridDim.x * blockDim.x) {
-        const float *p = D + mu * coord_step;
+    auto one = [&](const float (&x)[R]) {
         double mean = 0.0;
-        for (uint32_t i = 0; i < R; ++i) mean += (double)p[(uint64_t)i * replica_step];
+#pragma unroll
+        for (int i = 0; i < R; ++i) mean += (double)x[i];
         mean /= (double)R;
         double var = 0.0;
-        for (uint32_t i = 0; i < R; ++i) {
-            const double e = (double)p[(uint64_t)i * replica_step] - mean;
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const double e = (double)x[i] - mean;
             var += e * e;
         }
         var /= (double)R;
         acc += var;
         mx = var > mx ? var : mx;
+    };
+    if constexpr (MAJOR == 0) {
+        for (uint64_t mu = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; mu < N;
+             mu += (uint64_t)gridDim.x * blockDim.x) {
+            float x[R];
+            load_replicas<R>(D + mu * R, x);
+            one(x);
+        }
+    } else {
+        const uint64_t n4 = (N + 3) / 4;
+        for (uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n4;
+             q += (uint64_t)gridDim.x * blockDim.x) {
+            float4 r4[R];
+#pragma unroll
+            for (int i = 0; i < R; ++i) r4[i] = __ldcs(reinterpret_cast<const float4 *>(D + (uint64_t)i * stride) + q);
+            const uint64_t left = N - 4 * q;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if ((uint64_t)c < left) {
+                    float x[R];
+#pragma unroll
+                    for (int i = 0; i < R; ++i) x[i] = reinterpret_cast<const float *>(&r4[i])[c];
+                    one(x);
+                }
+            }
+        }
     }
     for (int d = 16; d > 0; d >>= 1) {
         acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
@@ -265,6 +332,22 @@ __global__ void spread_kernel(const float *D, uint32_t R, uint64_t coord_step, u
             atomicMax(reinterpret_cast<unsigned long long *>(out + 1),
                       (unsigned long long)__double_as_longlong(mx));
         }
+    }
+}
+
+typedef void (*spread_fn)(const float *, uint64_t, uint64_t, double *);
+template <int MAJOR>
+static spread_fn spread_for(uint32_t R)
+{
+    switch (R) {
+    case 1: return spread_kernel<1, MAJOR>;   case 2: return spread_kernel<2, MAJOR>;
+    case 3: return spread_kernel<3, MAJOR>;   case 4: return spread_kernel<4, MAJOR>;
+    case 5: return spread_kernel<5, MAJOR>;   case 6: return spread_kernel<6, MAJOR>;
+    case 7: return spread_kernel<7, MAJOR>;   case 8: return spread_kernel<8, MAJOR>;
+    case 9: return spread_kernel<9, MAJOR>;   case 10: return spread_kernel<10, MAJOR>;
+    case 11: return spread_kernel<11, MAJOR>; case 12: return spread_kernel<12, MAJOR>;
+    case 13: return spread_kernel<13, MAJOR>; case 14: return spread_kernel<14, MAJOR>;
+    case 15: return spread_kernel<15, MAJOR>; default: return spread_kernel<16, MAJOR>;
     }
 }
 
@@ -475,18 +558,21 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     // unless a flag asks for another kernel.  1B layout, tau = 4, ms per step, pipelined
     // against owner: p = 0.01 21.6 / 20.7, 0.05 23.4 / 22.7, 0.1 26.2 / 23.9, 0.25 30.9 / 25.6,
     // 0.5 37.4 / 29.0; tau = 0: 20.8 to 24.4 / 20.5 to 20.7 at every p.
+    // E4M3 exchange, the eager estimate and NAdamW: the kernels' general form.  The owner
+    // kernel carries that form's optimizer code four times over (once per unit of a
+    // group) and loses more to it than the pipelined kernel does (1B layout, NAdamW: 30.1
+    // against 24.1 ms per step), so the general form stays with the pipelined kernel.
+    const bool general = h->wire == 2u || h->correction == ASYNCMESH_CORRECTION_EAGER ||
+                         h->optimizer == ASYNCMESH_OPT_NADAMW;
     const bool owner_asked = (cfg->flags & ASYNCMESH_FLAG_OWNER_KERNEL) != 0;
     const bool owner_default =
-        !(cfg->flags & (ASYNCMESH_FLAG_DIRECT_KERNEL | ASYNCMESH_FLAG_PIPELINED_KERNEL)) &&
+        !general && !(cfg->flags & (ASYNCMESH_FLAG_DIRECT_KERNEL | ASYNCMESH_FLAG_PIPELINED_KERNEL)) &&
         (h->mode == kCompact || (h->mode == kSync && cfg->p <= 0.8));
     if (R <= 4 && h->mode != kDense && (owner_asked || owner_default)) {
         const double mean = 128.0 * kOwnerV * cfg->p, sd = std::sqrt(mean * (1.0 - cfg->p));
         h->pipelined = h->mode == kSync ? 6 : (mean + 4.0 * sd <= (double)kOwnerEntriesFew ? 4 : 5);
     }
 
-    // E4M3 exchange, the eager estimate and NAdamW: the kernels' general form
-    const bool general = h->wire == 2u || h->correction == ASYNCMESH_CORRECTION_EAGER ||
-                         h->optimizer == ASYNCMESH_OPT_NADAMW;
 
     auto bail = [&](int code, const char *what) {
         release_all(h);
@@ -555,6 +641,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
 
     // persistent grid: every SM filled to the kernel's occupancy
+    h->general = general;
     h->kernel = pick_kernel(R, h->mode, h->pipelined, general, S);
     int sms = 0, per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
@@ -732,7 +819,8 @@ extern "C" int asyncmesh_step(asyncmesh *h, const float *const *grads)
     return asyncmesh_step_ex(h, grads, -1.0, -1.0);
 }
 
-extern "C" int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host)
+extern "C" int asyncmesh_step_host_ex(asyncmesh *h, const float *const *grads_host,
+                                      double ema_beta_t, double lr_t)
 {
     if (!h || !grads_host) return fail(ASYNCMESH_ERR_INVALID_ARG, "step_host: NULL argument");
     DeviceScope scope(h->device);
@@ -744,11 +832,18 @@ extern "C" int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host)
             if (!h->gstage[s]) return fail(ASYNCMESH_ERR_OOM, "step_host: out of device memory (staging)");
             CU_TRY(cudaMemsetAsync(h->gstage[s], 0, bytes, h->stream));
         }
+        // one copy per replica row (a 2-D copy would cap the row at the device's largest pitch)
         const size_t n = h->numel[s] * sizeof(float);
-        CU_TRY(cudaMemcpy2DAsync(h->gstage[s], h->stride[s] * sizeof(float), grads_host[s], n, n,
-                                 h->R, cudaMemcpyHostToDevice, h->stream));
+        for (uint32_t i = 0; i < h->R; ++i)
+            CU_TRY(cudaMemcpyAsync(h->gstage[s] + (uint64_t)i * h->stride[s], grads_host[s] + (uint64_t)i * h->numel[s],
+                                   n, cudaMemcpyHostToDevice, h->stream));
     }
-    return launch_step(h, h->gstage.data(), -1.0, -1.0);
+    return launch_step(h, h->gstage.data(), ema_beta_t, lr_t);
+}
+
+extern "C" int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host)
+{
+    return asyncmesh_step_host_ex(h, grads_host, -1.0, -1.0);
 }
 
 // ---------------------------------------------------------------------------
@@ -913,9 +1008,11 @@ extern "C" int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *o
     if (!h || !out_host || stage >= h->S)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "consensus_error: bad handle, stage or output");
     DeviceScope scope(h->device);
+    int rc = check_status(h, "consensus_error");
+    if (rc != ASYNCMESH_OK) return rc;
     const StageDesc &d = h->sd[stage];
     CU_TRY(cudaMemsetAsync(h->scratch, 0, sizeof(double), h->stream));
-    consensus_kernel<<<grid_for(d.N, 256), 256, 0, h->stream>>>(d.W, h->R, d.stride, d.N, h->scratch);
+    consensus_for(h->R)<<<grid_for((d.N + 3) / 4, 256), 256, 0, h->stream>>>(d.W, d.stride, d.N, h->scratch);
     CU_TRY(cudaGetLastError());
     CU_TRY(cudaMemcpyAsync(out_host, h->scratch, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
     CU_TRY(cudaStreamSynchronize(h->stream));
@@ -928,13 +1025,15 @@ extern "C" int asyncmesh_ema_variance(asyncmesh *h, uint32_t stage, double *mean
     if (!h || !mean_host || !max_host || stage >= h->S)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "ema_variance: bad handle, stage or output");
     DeviceScope scope(h->device);
+    int rc = check_status(h, "ema_variance");
+    if (rc != ASYNCMESH_OK) return rc;
     const StageDesc &d = h->sd[stage];
     // d is coordinate-major [stride][R] except with the dense ring ([R][stride])
-    const uint64_t coord_step = h->mode == kDense ? 1 : h->R;
-    const uint64_t replica_step = h->mode == kDense ? d.stride : 1;
     CU_TRY(cudaMemsetAsync(h->scratch, 0, 2 * sizeof(double), h->stream));
-    spread_kernel<<<grid_for(d.N, 256), 256, 0, h->stream>>>(d.D, h->R, coord_step, replica_step, d.N,
-                                                             h->scratch);
+    if (h->mode == kDense)
+        spread_for<1>(h->R)<<<grid_for((d.N + 3) / 4, 256), 256, 0, h->stream>>>(d.D, d.stride, d.N, h->scratch);
+    else
+        spread_for<0>(h->R)<<<grid_for(d.N, 256), 256, 0, h->stream>>>(d.D, d.stride, d.N, h->scratch);
     CU_TRY(cudaGetLastError());
     double out[2];
     CU_TRY(cudaMemcpyAsync(out, h->scratch, sizeof out, cudaMemcpyDeviceToHost, h->stream));
@@ -948,6 +1047,22 @@ extern "C" int asyncmesh_step_count(const asyncmesh *h, uint64_t *t)
 {
     if (!h || !t) return fail(ASYNCMESH_ERR_INVALID_ARG, "step_count: NULL argument");
     *t = h->t;
+    return ASYNCMESH_OK;
+}
+
+extern "C" int asyncmesh_kernel_name(const asyncmesh *h, char *buf, size_t cap)
+{
+    if (!h || !buf || cap == 0) return fail(ASYNCMESH_ERR_INVALID_ARG, "kernel_name: NULL argument");
+    const char *mode = h->mode == kSync ? "sync" : (h->mode == kDense ? "dense" : "compact");
+    const char *form = h->general ? " general" : "";
+    switch (h->pipelined) {
+    case 0: snprintf(buf, cap, "direct R=%u %s%s", h->R, mode, form); break;
+    case 1: snprintf(buf, cap, "pipelined R=%u %s wide%s", h->R, mode, form); break;
+    case 2: case 3: snprintf(buf, cap, "pipelined R=%u %s narrow%s", h->R, mode, form); break;
+    case 4: snprintf(buf, cap, "owner R=%u %s entries=%d%s", h->R, mode, kOwnerEntriesFew, form); break;
+    case 5: snprintf(buf, cap, "owner R=%u %s entries=%d%s", h->R, mode, kOwnerEntriesMany, form); break;
+    default: snprintf(buf, cap, "owner R=%u %s%s", h->R, mode, form);
+    }
     return ASYNCMESH_OK;
 }
 

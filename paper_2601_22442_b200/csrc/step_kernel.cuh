@@ -168,12 +168,29 @@ __device__ __forceinline__ void adamw_group(const StepParams &P, const float (&w
         if (P.nesterov != 0u) {
             // NAdamW (Appendix B.1): gradient part and (uncorrected) momentum part over
             // the same denominator, weighted by the momentum schedule's cg and cm
+            float vlo = vh[0], vhi = vh[0], alo = fminf(fabsf(g[0]), fabsf(m[0])),
+                  ahi = fmaxf(fabsf(g[0]), fabsf(m[0]));
+#pragma unroll
+            for (int c = 1; c < NC; ++c) {
+                vlo = fminf(vlo, vh[c]);
+                vhi = fmaxf(vhi, vh[c]);
+                alo = fminf(alo, fminf(fabsf(g[c]), fabsf(m[c])));
+                ahi = fmaxf(ahi, fmaxf(fabsf(g[c]), fabsf(m[c])));
+            }
+            const bool inrange = P.eps_inrange != 0u && vlo >= kSqrtLo && vhi <= kSqrtHi &&
+                                 alo >= kDivNumLo && ahi <= kDivNumHi;
 #pragma unroll
             for (int c = 0; c < NC; ++c) {
-                const float den = __fadd_rn(__fsqrt_rn(vh[c]), P.eps);
+                float ug, um;
+                if (inrange) {
+                    const float den = __fadd_rn(sqrt_rn_inrange(vh[c]), P.eps);
+                    ug = div_rn_inrange(g[c], den);
+                    um = div_rn_inrange(m[c], den);
+                } else {
+                    ug = adam_quotient_anyrange(g[c], vh[c], P.eps);
+                    um = adam_quotient_anyrange(m[c], vh[c], P.eps);
+                }
                 const float decayed = __fsub_rn(w[c], __fmul_rn(P.lrwd, w[c]));
-                const float ug = __fdiv_rn(g[c], den);
-                const float um = __fdiv_rn(m[c], den);
                 what[c] = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug)), __fmul_rn(P.cm, um));
             }
             return;

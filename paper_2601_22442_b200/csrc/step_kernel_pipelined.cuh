@@ -399,6 +399,9 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
                         }
                     }
                 }
+                // every lane has read w^{t-1} of the coordinate it adopted (another lane's)
+                // before any lane overwrites that row in the dense loop below
+                __syncwarp();
             }
 
             // ---- dense arithmetic, one replica (= one pipeline unit) at a time ----

@@ -203,6 +203,8 @@ def test_nadamw(tau, p):
     run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
              flags=binding.FLAG_DIRECT_KERNEL)
     run_case(6, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp)   # pipelined kernel
+    run_case(4, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
+             flags=binding.FLAG_OWNER_KERNEL)
 
 
 @pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (3, 0.4)])
@@ -231,7 +233,7 @@ def test_fp8_exchange(tau, p):
     run_case(3, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="fp8",
              flags=binding.FLAG_DIRECT_KERNEL)
     run_case(4, [6000], p, tau, 0.9, steps=3 * tau + 5, exchange="fp8",
-             flags=binding.FLAG_PIPELINED_KERNEL)
+             flags=binding.FLAG_OWNER_KERNEL)
     ref = oracle.Oracle(4, [6000, 1024 + 9], p=p, tau=tau, ema_beta=0.9, exchange="bf16", **HP)
     for s, n in enumerate([6000, 1024 + 9]):
         ref.init_params(s, si.init_weights_host(0x1217, s, 0, n))
@@ -282,7 +284,7 @@ def test_eager_staleness_estimate(p, tau, K):
     run_case(3, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
              flags=binding.FLAG_DIRECT_KERNEL)
     run_case(4, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
-             flags=binding.FLAG_PIPELINED_KERNEL)
+             flags=binding.FLAG_OWNER_KERNEL)
     if 0 < p < 1 and tau:
         run_case(3, [7000], p, tau, 0.4, steps=steps, avg_interval=K, correction="eager",
                  flags=binding.FLAG_DENSE_RING)
@@ -415,13 +417,34 @@ def test_step_host_equals_step():
         hg = [si.grads_host(2, t, s, 3, 0, n) for s, n in enumerate(numel)]
         for s, n in enumerate(numel):
             bufs[s][:, :n].copy_(torch.from_numpy(hg[s]))
-        a.step(bufs)
         pinned = [torch.from_numpy(x).pin_memory() for x in hg]
-        b.step_host(pinned)
+        if t % 2:
+            a.step(bufs)
+            b.step_host(pinned)
+        else:           # the per-step scalars reach the host-gradient form too
+            a.step(bufs, ema_beta_t=0.3, lr_t=1e-4)
+            b.step_host(pinned, ema_beta_t=0.3, lr_t=1e-4)
         b.status()
     for s in range(2):
         for name in STATE_NAMES:
             assert np.array_equal(a.get(s, name), b.get(s, name))
+
+
+def test_kernel_name_tells_which_kernel_runs():
+    from paper_2601_22442_b200 import binding
+    mk = lambda R, p, tau, flags=0, **kw: am().AsyncMesh(R, [5000], p=p, tau=tau, ema_beta=0.9, flags=flags,
+                                                          **dict(HP, **kw)).kernel_name()
+    assert mk(4, 0.05, 2) == "owner R=4 compact entries=32"
+    assert mk(4, 0.3, 2) == "owner R=4 compact entries=128"
+    assert mk(3, 0.3, 0) == "owner R=3 sync"
+    assert mk(8, 0.05, 2) == "pipelined R=8 compact wide"
+    assert mk(8, 0.3, 2) == "pipelined R=8 compact narrow"
+    assert mk(4, 0.05, 2, binding.FLAG_PIPELINED_KERNEL) == "pipelined R=4 compact wide"
+    assert mk(4, 0.05, 2, binding.FLAG_DIRECT_KERNEL) == "direct R=4 compact"
+    assert mk(4, 1.0, 2) == "direct R=4 dense"
+    assert mk(4, 1.0, 0) == "direct R=4 sync"
+    assert mk(4, 0.05, 2, optimizer="nadamw") == "pipelined R=4 compact wide general"
+    assert mk(4, 0.05, 2, binding.FLAG_OWNER_KERNEL, optimizer="nadamw") == "owner R=4 compact entries=32 general"
 
 
 def test_init_from_device_tensor_and_bad_state():

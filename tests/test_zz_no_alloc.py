@@ -35,8 +35,11 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
             want = g.consensus_error(s)
             ptr, stride = g.lookahead_weights(s, 0)
             before = torch.cuda.memory_allocated()
+            free_before = torch.cuda.mem_get_info()[0]      # the driver's own count of free bytes
             got = pkg.asyncmesh_consensus_error_noalloc(ptr, R, n, stride, device=0, stream=stream)
             assert torch.cuda.memory_allocated() == before
+            if call == 1:   # module loaded, scratch address known: a raw cudaMalloc would show here
+                assert torch.cuda.mem_get_info()[0] == free_before
             assert want > 0
             # both reduce in double; only the summation order differs
             assert abs(got - want) <= 1e-9 * want, (call, s, got, want)
