@@ -27,7 +27,7 @@ KernelChoice pick_pipelined_few_common(uint32_t R, int shape, uint32_t S);     /
 KernelChoice pick_pipelined_few_general(uint32_t R, int shape, uint32_t S);
 KernelChoice pick_pipelined_many_common(uint32_t R, int shape, uint32_t S);    // R = 9..16
 KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S);
-// Owner kernel (R = 1..4).  mode: kCompact or kSync; entries: ring / d entries per group
+// Owner kernel (R = 1..4; R = 5..8 for kSync only).  mode: kCompact or kSync; entries: ring / d entries per group
 // of 256 coordinates fetched ahead (kOwnerEntriesFew or kOwnerEntriesMany).
 // Shape, measured on the 1B layout (R = 4, p = 0.05, ms per step): one replica row per
 // unit and 8 coordinates per lane (1 KB contiguous per array row and request) 22.7;
@@ -36,7 +36,8 @@ KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S);
 constexpr int kOwnerStages = 3;
 constexpr int kOwnerV = 2;
 constexpr int kOwnerEntriesFew = 32, kOwnerEntriesMany = 128;
-constexpr int owner_ru(int) { return 1; }
+// replica rows per unit: one up to four replicas; with more, two where that divides R (8 KB units)
+constexpr int owner_ru(int R) { return (R > 4 && R % 2 == 0) ? 2 : 1; }
 KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S);
 KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S);
 

@@ -230,7 +230,7 @@ __device__ __forceinline__ float div_by_replicas(const StepParams &P, float a)
 
 // MODE kCompact (tau >= 1) or kSync (tau = 0).
 template <int R, int RU, int V, int NST, int E, int MODE, bool GEN>
-__global__ void __launch_bounds__(kOwnerThreads, kOwnerBlocksPerSM)
+__global__ void __launch_bounds__(kOwnerThreads, R <= 4 ? kOwnerBlocksPerSM : 2)
 asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
 {
     static_assert(MODE == kCompact || MODE == kSync, "compact ring or synchronous");
@@ -395,7 +395,10 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
             if constexpr (UPG > 1) unit(std::integral_constant<int, 1>{});
             if constexpr (UPG > 2) unit(std::integral_constant<int, 2>{});
             if constexpr (UPG > 3) unit(std::integral_constant<int, 3>{});
-            static_assert(UPG <= 4, "at most four units per group");
+            if constexpr (UPG > 4) unit(std::integral_constant<int, 4>{});
+            if constexpr (UPG > 5) unit(std::integral_constant<int, 5>{});
+            if constexpr (UPG > 6) unit(std::integral_constant<int, 6>{});
+            static_assert(UPG <= 7, "at most seven units per group");
 
             if constexpr (MODE == kCompact) {
                 // ---- snapshot of the local iterate on S^t (Section 3.1) ------------------

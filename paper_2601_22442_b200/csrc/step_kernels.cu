@@ -1,7 +1,7 @@
 // Instantiations of the step kernels.  Compiled nine times, -DAM_PART=0..8:
 // 0 direct kernel R = 1..8; 1 direct kernel R = 9..16, common form; 2 the same,
 // general form; 3 / 4 pipelined kernel R = 1..8, common / general form; 5 / 6
-// pipelined kernel R = 9..16, common / general form; 7 / 8 owner kernel R = 1..4,
+// pipelined kernel R = 9..16, common / general form; 7 / 8 owner kernel R = 1..8,
 // common / general form.
 #include "kernel_table.cuh"
 
@@ -101,6 +101,11 @@ KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S)
     case 2: return owner<2>(mode, entries, S);
     case 3: return owner<3>(mode, entries, S);
     case 4: return owner<4>(mode, entries, S);
+    // five to eight replicas: the synchronous mode only (with the ring the pipelined kernel is as fast or faster)
+    case 5: return mode == kSync ? owner_as<5, 1, kSync>(S) : KernelChoice();
+    case 6: return mode == kSync ? owner_as<6, 1, kSync>(S) : KernelChoice();
+    case 7: return mode == kSync ? owner_as<7, 1, kSync>(S) : KernelChoice();
+    case 8: return mode == kSync ? owner_as<8, 1, kSync>(S) : KernelChoice();
     default: return KernelChoice();
     }
 }

@@ -437,6 +437,8 @@ def test_kernel_name_tells_which_kernel_runs():
     assert mk(4, 0.05, 2) == "owner R=4 compact entries=32"
     assert mk(4, 0.3, 2) == "owner R=4 compact entries=128"
     assert mk(3, 0.3, 0) == "owner R=3 sync"
+    assert mk(8, 0.3, 0) == "owner R=8 sync" and mk(7, 0.05, 0) == "owner R=7 sync"
+    assert mk(9, 0.3, 0) == "pipelined R=9 sync narrow"
     assert mk(8, 0.05, 2) == "pipelined R=8 compact wide"
     assert mk(8, 0.3, 2) == "pipelined R=8 compact narrow"
     assert mk(4, 0.05, 2, binding.FLAG_PIPELINED_KERNEL) == "pipelined R=4 compact wide"
