@@ -317,7 +317,10 @@ int asyncmesh_min_bytes_last_step(const asyncmesh *h, uint64_t *bytes);
 int asyncmesh_status(asyncmesh *h);
 
 /* Run the device's Philox-4x32-10 on n (counter, key) pairs: ctr_host [n][4],
- * key_host [n][2], out_host [n][4], all uint32 in host memory.  Test hook. */
+ * key_host [n][2], out_host [n][4], all uint32 in host memory.  Test hook: it has no
+ * handle, so its three temporary device buffers come from cudaMalloc / cudaFree, not
+ * from a handle's allocator callbacks.  (The generator is the published one, Salmon et
+ * al., SC'11; Section 2.3 of the paper only asks for a randomly sampled subset.) */
 int asyncmesh_debug_philox(int device, const uint32_t *ctr_host,
                            const uint32_t *key_host, uint32_t *out_host, uint64_t n);
 
