@@ -57,7 +57,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", choices=["native", "reference"], default="native")
     ap.add_argument("--workload", default="llama1b",
-                    help="toy | llama125m | llama350m | llama1b")
+                    help="toy | llama125m | llama350m | llama1b | profile | profile8")
     ap.add_argument("--p", type=float, default=None)
     ap.add_argument("--tau", type=int, default=None)
     ap.add_argument("--no-e2e", action="store_true")

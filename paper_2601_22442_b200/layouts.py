@@ -58,6 +58,7 @@ def workloads() -> Dict[str, dict]:
                           tau=4, steps=50),
         # small case for profiler captures: larger than L2, a few GB on the device
         "profile": dict(R=4, numel=[1 << 24, 1 << 24], tau=4, steps=8),
+        "profile8": dict(R=8, numel=[1 << 23, 1 << 23], tau=4, steps=8),     # the same bytes, eight replicas
         "llama1b": dict(R=4, numel=llama_stage_numel(2048, 16, 5632, 32000, 8, False),
                         tau=4, steps=20),
     }

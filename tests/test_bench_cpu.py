@@ -112,3 +112,11 @@ def test_coordinate_shards_of_two_ranks_tile_every_stage():
         coordinate_shard([1000], 0, 2)
     with pytest.raises(ValueError):
         coordinate_shard([5000], 0, 2, align=6)
+
+
+def test_traffic_ratio_is_looked_up_by_kernel_name_and_p():
+    import bench
+    assert bench.measured_traffic_ratio("owner R=4 compact entries=32", 0.05) == pytest.approx(1.035)
+    assert bench.measured_traffic_ratio("pipelined R=8 compact wide", 0.05) == pytest.approx(1.012)
+    assert bench.measured_traffic_ratio("owner R=4 compact entries=32", 0.07) is None      # no capture at that p
+    assert bench.measured_traffic_ratio("no such kernel", 0.05) is None
