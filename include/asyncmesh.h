@@ -194,9 +194,14 @@ int asyncmesh_step_ex(asyncmesh *h, const float *const *grads,
 /*
  * The same step with gradients in HOST memory: grads_host[j] is [R][numel_j]
  * fp32, rows contiguous (no padding).  They are copied into library-owned
- * device staging buffers (allocated on the first call) on the handle's
- * stream, then the step runs.  Pinned host memory makes the copies
- * asynchronous; pageable memory works and is slower.
+ * device staging buffers (allocated on the first call), stage by stage, on a
+ * stream of the library's own (created on the first call), and the step runs as
+ * one launch per stage on the handle's stream, each as soon as its stage's
+ * gradients have arrived: the kernels of all but the last stage run while later
+ * stages are still being copied.  The result is the same as that of
+ * asyncmesh_step.  The host buffers may be reused once the handle's stream has
+ * passed the step.  Pinned host memory makes the copies asynchronous; pageable
+ * memory works and is slower.
  */
 int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host);
 int asyncmesh_step_host_ex(asyncmesh *h, const float *const *grads_host,

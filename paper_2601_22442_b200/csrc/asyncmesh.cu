@@ -90,6 +90,10 @@ struct asyncmesh {
     std::vector<void *> owned;        // everything obtained from the allocator
 
     StageDesc *sd_dev = nullptr;
+    StageDesc *sd_single_dev = nullptr;   // the same table with chunk_begin = 0: one-stage launches
+    cudaStream_t copy_stream = nullptr;   // asyncmesh_step_host: gradient copies, overlapping the kernels
+    std::vector<cudaEvent_t> ev_ready, ev_done;   // per stage: gradients copied / kernel done with them
+    std::vector<char> done_recorded;
     unsigned int *cursors = nullptr;  // [n_slots][S]
     int *status = nullptr;
     double *scratch = nullptr;        // a few doubles for reductions
@@ -628,12 +632,17 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         }
     }
     h->sd_dev = (StageDesc *)zalloc(S * sizeof(StageDesc));
+    h->sd_single_dev = (StageDesc *)zalloc(S * sizeof(StageDesc));
     h->cursors = (unsigned int *)zalloc((size_t)(h->n_slots + 1) * S * sizeof(unsigned int));
     h->status = (int *)zalloc(256);
     h->scratch = (double *)zalloc(256);
-    if (!h->sd_dev || !h->cursors || !h->status || !h->scratch)
+    if (!h->sd_dev || !h->sd_single_dev || !h->cursors || !h->status || !h->scratch)
         return bail(ASYNCMESH_ERR_OOM, "out of device memory (tables)");
+    std::vector<StageDesc> single(h->sd);
+    for (StageDesc &d1 : single) d1.chunk_begin = 0;
     if (cudaMemcpyAsync(h->sd_dev, h->sd.data(), S * sizeof(StageDesc), cudaMemcpyHostToDevice,
+                        h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(h->sd_single_dev, single.data(), S * sizeof(StageDesc), cudaMemcpyHostToDevice,
                         h->stream) != cudaSuccess ||
         cudaStreamSynchronize(h->stream) != cudaSuccess) {
         const char *msg = cudaGetErrorString(cudaGetLastError());
@@ -677,6 +686,12 @@ extern "C" int asyncmesh_destroy(asyncmesh *h)
     if (!h) return ASYNCMESH_OK;
     DeviceScope scope(h->device);
     cudaStreamSynchronize(h->stream);
+    if (h->copy_stream) {
+        cudaStreamSynchronize(h->copy_stream);
+        for (cudaEvent_t e : h->ev_ready) cudaEventDestroy(e);
+        for (cudaEvent_t e : h->ev_done) cudaEventDestroy(e);
+        cudaStreamDestroy(h->copy_stream);
+    }
     release_all(h);
     delete h;
     return ASYNCMESH_OK;
@@ -723,7 +738,10 @@ extern "C" int asyncmesh_row_stride(const asyncmesh *h, uint32_t stage, uint64_t
 // the step
 // ---------------------------------------------------------------------------
 
-static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_t, double lr_t)
+// stage_ready: NULL, or one event per stage that the stage's gradients wait for; the step then
+// runs as one launch per stage, each as soon as its gradients are there.
+static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_t, double lr_t,
+                       const cudaEvent_t *stage_ready = nullptr)
 {
     if (ema_beta_t > 1.0) return fail(ASYNCMESH_ERR_INVALID_ARG, "step: ema_beta_t = %g above 1", ema_beta_t);
     StepParams P;
@@ -743,6 +761,8 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.status = h->status;
     P.S = h->S;
     P.total_chunks = h->total_chunks;
+    P.cursor_S = h->S;
+    P.s_base = 0;
     P.step = (uint32_t)t;
     // averaging rounds are the steps K, 2K, ...; in between the step is purely local
     const bool round = (t % h->K) == 0;
@@ -792,8 +812,27 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
         CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
                                h->S * sizeof(unsigned int), h->stream));
 
-    h->kernel.fn<<<h->grid, h->kernel.threads, h->kernel.smem, h->stream>>>(P);
-    CU_TRY(cudaGetLastError());
+    if (!stage_ready) {
+        h->kernel.fn<<<h->grid, h->kernel.threads, h->kernel.smem, h->stream>>>(P);
+        CU_TRY(cudaGetLastError());
+    } else {
+        const uint32_t wpb = (uint32_t)h->kernel.threads / 32;
+        for (uint32_t s = 0; s < h->S; ++s) {
+            StepParams Q = P;
+            Q.stages = h->sd_single_dev + s;
+            Q.S = 1;
+            Q.s_base = s;
+            Q.total_chunks = h->sd[s].n_chunks;
+            Q.G[0] = grads[s];
+            int grid = (int)((Q.total_chunks + wpb - 1) / wpb);
+            if (grid > h->grid) grid = h->grid;
+            CU_TRY(cudaStreamWaitEvent(h->stream, stage_ready[s], 0));
+            h->kernel.fn<<<grid, h->kernel.threads, h->kernel.smem, h->stream>>>(Q);
+            CU_TRY(cudaGetLastError());
+            CU_TRY(cudaEventRecord(h->ev_done[s], h->stream));
+            h->done_recorded[s] = 1;
+        }
+    }
     h->t = t;
     h->mu_product = mu_product;
 
@@ -826,21 +865,38 @@ extern "C" int asyncmesh_step_host_ex(asyncmesh *h, const float *const *grads_ho
 {
     if (!h || !grads_host) return fail(ASYNCMESH_ERR_INVALID_ARG, "step_host: NULL argument");
     DeviceScope scope(h->device);
-    for (uint32_t s = 0; s < h->S; ++s) {
+    for (uint32_t s = 0; s < h->S; ++s)
         if (!grads_host[s]) return fail(ASYNCMESH_ERR_INVALID_ARG, "step_host: grads_host[%u] is NULL", s);
+    if (!h->copy_stream) {   // first call: a stream for the copies and the events that tie it to the kernels
+        CU_TRY(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+        h->ev_ready.assign(h->S, nullptr);
+        h->ev_done.assign(h->S, nullptr);
+        h->done_recorded.assign(h->S, 0);
+        for (uint32_t s = 0; s < h->S; ++s) {
+            CU_TRY(cudaEventCreateWithFlags(&h->ev_ready[s], cudaEventDisableTiming));
+            CU_TRY(cudaEventCreateWithFlags(&h->ev_done[s], cudaEventDisableTiming));
+        }
+    }
+    // Stage by stage on the copy stream: wait until the previous step's kernel is done with the
+    // stage's staging buffer, copy, signal.  The kernels (one launch per stage, on the handle's
+    // stream) start as their gradients arrive, so all but the last stage's compute hides behind
+    // the copies of the stages after it.
+    for (uint32_t s = 0; s < h->S; ++s) {
         if (!h->gstage[s]) {
             const size_t bytes = (size_t)h->R * h->stride[s] * sizeof(float);
             h->gstage[s] = (float *)dev_alloc(h, bytes);
             if (!h->gstage[s]) return fail(ASYNCMESH_ERR_OOM, "step_host: out of device memory (staging)");
-            CU_TRY(cudaMemsetAsync(h->gstage[s], 0, bytes, h->stream));
+            CU_TRY(cudaMemsetAsync(h->gstage[s], 0, bytes, h->copy_stream));
         }
+        if (h->done_recorded[s]) CU_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_done[s], 0));
         // one copy per replica row (a 2-D copy would cap the row at the device's largest pitch)
         const size_t n = h->numel[s] * sizeof(float);
         for (uint32_t i = 0; i < h->R; ++i)
             CU_TRY(cudaMemcpyAsync(h->gstage[s] + (uint64_t)i * h->stride[s], grads_host[s] + (uint64_t)i * h->numel[s],
-                                   n, cudaMemcpyHostToDevice, h->stream));
+                                   n, cudaMemcpyHostToDevice, h->copy_stream));
+        CU_TRY(cudaEventRecord(h->ev_ready[s], h->copy_stream));
     }
-    return launch_step(h, h->gstage.data(), ema_beta_t, lr_t);
+    return launch_step(h, h->gstage.data(), ema_beta_t, lr_t, h->ev_ready.data());
 }
 
 extern "C" int asyncmesh_step_host(asyncmesh *h, const float *const *grads_host)

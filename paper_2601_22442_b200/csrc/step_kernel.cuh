@@ -77,7 +77,9 @@ struct StepParams {
     unsigned int *cursors;       // device [n_slots][S]            (compact only)
     int *status;                 // device status word
     const float *G[kMaxStages];  // gradients, [R][stride] each
-    uint32_t S, total_chunks;
+    uint32_t S, total_chunks;    // stages and warp chunks of THIS launch
+    uint32_t cursor_S, s_base;   // stages of the handle and the handle's index of this launch's stage 0:
+                                 // a launch may cover one stage only (host gradients arriving stage by stage)
     uint32_t step, cons_step;    // t and t - tau
     uint32_t produce;            // this step is an averaging round: S^t is snapshotted
     uint32_t consume;            // ... and the average launched at t - tau has arrived
@@ -291,7 +293,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
         if (lane == 0) {
             uint32_t b = 0;
             if (total) {
-                b = atomicAdd(&P.cursors[P.prod_slot * P.S + s], total);
+                b = atomicAdd(&P.cursors[P.prod_slot * P.cursor_S + P.s_base + s], total);
                 if (b > st.cap || total > st.cap - b) {   // slot full: drop loudly
                     b = kInvalidBase;
                     atomicExch(P.status, kStatusRingOverflow);

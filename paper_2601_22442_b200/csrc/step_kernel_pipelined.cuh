@@ -292,7 +292,7 @@ asyncmesh_step_kernel_pipelined(const __grid_constant__ StepParams P)
         if (lane == 0) {
             uint32_t b = 0;
             if (total) {
-                b = atomicAdd(&P.cursors[P.prod_slot * P.S + s], total);
+                b = atomicAdd(&P.cursors[P.prod_slot * P.cursor_S + P.s_base + s], total);
                 if (b > st.cap || total > st.cap - b) {   // slot full: drop loudly
                     b = kInvalidBase;
                     atomicExch(P.status, kStatusRingOverflow);

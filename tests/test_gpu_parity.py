@@ -405,16 +405,20 @@ def test_coordinate_shards_equal_the_unsharded_stage(p, tau, flags):
         am().AsyncMesh(R, [100], p=p, tau=tau, ema_beta=0.9, coord_base=[6], **HP)
 
 
-def test_step_host_equals_step():
-    numel = [3000, 1025]
-    a = am().AsyncMesh(3, numel, p=0.2, tau=1, ema_beta=0.9, **HP)
-    b = am().AsyncMesh(3, numel, p=0.2, tau=1, ema_beta=0.9, **HP)
+@pytest.mark.parametrize("R,p,tau,flags", [(3, 0.2, 1, 0), (4, 0.05, 2, 0), (8, 0.05, 2, 0), (8, 0.3, 0, 0),
+                                           (4, 0.3, 2, 2), (4, 1.0, 2, 0), (5, 0.4, 2, 4)])
+def test_step_host_equals_step(R, p, tau, flags):
+    # host gradients: copied stage by stage on the library's own stream, one launch per stage as
+    # its gradients arrive -- the same state as the single launch on device gradients
+    numel = [3000, 1025, 5000]
+    a = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=0.9, flags=flags, **HP)
+    b = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=0.9, flags=flags, **HP)
     for s, n in enumerate(numel):
         w0 = si.init_weights_host(1, s, 0, n)
         a.init_params(s, w0); b.init_params(s, w0)
     bufs = a.empty_grads()
-    for t in range(1, 5):
-        hg = [si.grads_host(2, t, s, 3, 0, n) for s, n in enumerate(numel)]
+    for t in range(1, 2 * tau + 5):
+        hg = [si.grads_host(2, t, s, R, 0, n) for s, n in enumerate(numel)]
         for s, n in enumerate(numel):
             bufs[s][:, :n].copy_(torch.from_numpy(hg[s]))
         pinned = [torch.from_numpy(x).pin_memory() for x in hg]
@@ -424,10 +428,13 @@ def test_step_host_equals_step():
         else:           # the per-step scalars reach the host-gradient form too
             a.step(bufs, ema_beta_t=0.3, lr_t=1e-4)
             b.step_host(pinned, ema_beta_t=0.3, lr_t=1e-4)
-        b.status()
-    for s in range(2):
+        if t == 2:
+            b.status()
+    b.status()
+    for s in range(len(numel)):
         for name in STATE_NAMES:
-            assert np.array_equal(a.get(s, name), b.get(s, name))
+            assert np.array_equal(a.get(s, name), b.get(s, name)), (s, name)
+        assert np.array_equal(a.subset_mask(s, 3), b.subset_mask(s, 3))
 
 
 def test_kernel_name_tells_which_kernel_runs():
