@@ -1,7 +1,7 @@
 // Third form of the fused step, for few replicas (up to four; up to eight for tau = 0):
-// the lane that owns a coordinate
-// does all of its work, sparse part included, and nothing is handed from lane to
-// lane.  Same results as the other two kernels, bit for bit.
+// the lane that owns a coordinate does all of its work, sparse part included, and
+// nothing is handed from lane to lane.  Same results as the other two kernels, bit
+// for bit.
 //
 //  * A lane owns 4 V coordinates of a group of 128 V (V float4 per array row) and
 //    keeps the R replica values of each in registers: the stale replica average
