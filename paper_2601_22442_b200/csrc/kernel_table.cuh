@@ -33,7 +33,11 @@ KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S);
 // unit and 8 coordinates per lane (1 KB contiguous per array row and request) 22.7;
 // two rows per unit 23.0; 4 coordinates per lane (512-byte requests) 24.3 to 24.8 whatever
 // the rows per unit: the request size is worth 1 ms, also with nothing selected.
-constexpr int kOwnerStages = 3;
+// Stages of the copy pipeline: three with the ring; two for tau = 0, where nothing but the dense stream
+// is in flight (1B layout, tau = 0: 19.2 against 20.4 ms per step; 350M layout: 13.9 against 14.2; with the
+// ring two stages lose: 25.3 against 22.6 at p = 0.05, 23.1 against 20.7 at p = 0.01, also when the sparse
+// copies are tracked apart from the dense ones).
+constexpr int owner_stages(int mode) { return mode == kSync ? 2 : 3; }
 constexpr int kOwnerV = 2;
 constexpr int kOwnerEntriesFew = 32, kOwnerEntriesMany = 128;
 // replica rows per unit: one up to four replicas; with more, two where that divides R (8 KB units)

@@ -75,10 +75,10 @@ template <int R, int E, int MODE>
 static KernelChoice owner_as(uint32_t S)
 {
     KernelChoice c;
-    c.fn = asyncmesh_step_kernel_owner<R, owner_ru(R), kOwnerV, kOwnerStages, E, MODE, kGeneral>;
+    c.fn = asyncmesh_step_kernel_owner<R, owner_ru(R), kOwnerV, owner_stages(MODE), E, MODE, kGeneral>;
     c.threads = kOwnerThreads;
     c.smem = (size_t)pipe_table_bytes(S) +
-             (size_t)(kOwnerThreads / 32) * OwnerCfg<R, owner_ru(R), kOwnerV, E>::warp_bytes(kOwnerStages);
+             (size_t)(kOwnerThreads / 32) * OwnerCfg<R, owner_ru(R), kOwnerV, E>::warp_bytes(owner_stages(MODE));
     return c;
 }
 
