@@ -55,14 +55,6 @@ __device__ __forceinline__ void cp_async_replicas(uint32_t smem_addr, const floa
     }
 }
 
-// 32 bytes to a 32-byte aligned address in one request
-__device__ __forceinline__ void st_sector(float *p, const float (&x)[8])
-{
-    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]),
-                 "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7])
-                 : "memory");
-}
-
 // RU: replica rows per pipeline unit (divides R); V: float4 per lane, array row and unit;
 // E: coordinates per group whose ring and d entries are fetched ahead (further ones,
 // possible only when p is large for the E chosen, are read in place).

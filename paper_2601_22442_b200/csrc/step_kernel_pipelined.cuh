@@ -80,10 +80,25 @@ __device__ __forceinline__ void cp_async_wait()
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
+// 32 bytes to a 32-byte aligned address in one request
+__device__ __forceinline__ void st_sector(float *p, const float (&x)[8])
+{
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]),
+                 "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7])
+                 : "memory");
+}
+
 template <int R>
 __device__ __forceinline__ void store_replicas(float *p, const float (&x)[R])
 {
-    if constexpr (R % 4 == 0) {
+    if constexpr (R % 8 == 0) {   // whole 32-byte sectors (entries of 8 replicas are 32-byte aligned)
+#pragma unroll
+        for (int q = 0; q < R / 8; ++q) {
+            const float s8[8] = {x[8 * q], x[8 * q + 1], x[8 * q + 2], x[8 * q + 3],
+                                 x[8 * q + 4], x[8 * q + 5], x[8 * q + 6], x[8 * q + 7]};
+            st_sector(p + 8 * q, s8);
+        }
+    } else if constexpr (R % 4 == 0) {
 #pragma unroll
         for (int q = 0; q < R / 4; ++q)
             *reinterpret_cast<float4 *>(p + 4 * q) =
