@@ -73,7 +73,10 @@ struct OwnerCfg {
     static constexpr int kSparseBytes = E * kEntryFloats * 4;
     __host__ __device__ static constexpr int sparse_areas(int stages)
     {
-        return (stages + 2 * kUnitsPerGroup - 2) / kUnitsPerGroup;   // groups that can be in flight
+        // groups whose sparse data can be in shared memory at a time: the one being finished, the
+        // next, and those the copy side has entered beyond it (it runs stages - 1 units ahead of
+        // the next group's first unit, which is fetched before the finished group's sparse work)
+        return 2 + (stages - 1) / kUnitsPerGroup;
     }
     __host__ __device__ static constexpr int warp_bytes(int stages)
     {
@@ -277,6 +280,21 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                                                     lt, n_warps, consume);
     uint32_t rd = 0, wr = NST - 1;   // stage being consumed / being filled
     uint32_t sp_rd = 0;              // sparse area of the group being computed
+    // Moves the pipeline on by one unit: waits for the next unit's data, asks for the unit NST - 1 further on
+    // (CU: that unit's place in its group) and returns where this lane's part of the arrived unit is.
+    auto advance = [&](auto cu_tag) -> const unsigned char * {
+        constexpr int CU = decltype(cu_tag)::value;
+        cp_async_wait<NST - 2>();
+        owner_issue_unit<R, RU, V, E, NST, CU>(pf, P, sd, stage_base + wr * kUnitBytes, sparse_base, lane, lt,
+                                               n_warps, consume);
+        const unsigned char *slot = my + rd * kUnitBytes + lane * 16;
+        rd = (rd + 1 == NST) ? 0 : rd + 1;
+        wr = (wr + 1 == NST) ? 0 : wr + 1;
+        return slot;
+    };
+    // A group's first unit is fetched BEFORE the sparse work of the group before it, so that the copies keep
+    // flowing while that work runs; this is the very first one.
+    const unsigned char *first_slot = advance(std::integral_constant<int, (NST - 1) % UPG>{});
 
     uint32_t s = 0;
     for (uint32_t gc = blockIdx.x * wpb + warp; gc < P.total_chunks; gc += n_warps) {
@@ -351,12 +369,8 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
             float wn[R][NB], wo[R][NB];
             auto unit = [&](auto u_tag) {
                 constexpr int u = decltype(u_tag)::value;
-                cp_async_wait<NST - 2>();
-                owner_issue_unit<R, RU, V, E, NST, (u + NST - 1) % UPG>(pf, P, sd, stage_base + wr * kUnitBytes,
-                                                                        sparse_base, lane, lt, n_warps, consume);
-                const unsigned char *slot = my + rd * kUnitBytes + lane * 16;
-                rd = (rd + 1 == NST) ? 0 : rd + 1;
-                wr = (wr + 1 == NST) ? 0 : wr + 1;
+                const unsigned char *slot =
+                    u == 0 ? first_slot : advance(std::integral_constant<int, (u + NST - 1) % UPG>{});
 #pragma unroll
                 for (int ii = 0; ii < RU; ++ii) {
                     const int i = u * RU + ii;
@@ -394,6 +408,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
             if constexpr (UPG > 5) unit(std::integral_constant<int, 5>{});
             if constexpr (UPG > 6) unit(std::integral_constant<int, 6>{});
             static_assert(UPG <= 7, "at most seven units per group");
+            first_slot = advance(std::integral_constant<int, (NST - 1) % UPG>{});   // the next group's, see above
 
             if constexpr (MODE == kCompact) {
                 // ---- snapshot of the local iterate on S^t (Section 3.1) ------------------
