@@ -69,6 +69,13 @@ extern "C" {
                                            is (up to four replicas; it is the default there for
                                            the compact ring and for tau = 0, this flag only extends
                                            it to subsets the dense ring would otherwise serve)  */
+#define ASYNCMESH_FLAG_TRACK_CONSENSUS 512u /* every step also accumulates the consensus error of each stage
+                                              (Section 3.3) from the final weights the step kernel holds in
+                                              registers: asyncmesh_consensus_error then returns the value of
+                                              the last step without another pass over the weights.  Honoured
+                                              where the owner kernel runs in its common form (up to four
+                                              replicas; up to eight for tau = 0); elsewhere the flag changes
+                                              nothing and the call makes its own pass as usual           */
 #define ASYNCMESH_FLAG_BF16_EXCHANGE 16u /* the subset is exchanged in bfloat16 (the paper's
                                            quantisation study): every snapshot value entering the
                                            replica average is first rounded to bfloat16 (nearest
@@ -251,7 +258,11 @@ int asyncmesh_subset_mask(asyncmesh *h, uint32_t stage, uint64_t step,
 
 /*
  * Consensus error of a stage, sum_i ||w_i - wbar||^2 (Section 3.3), reduced on
- * the device in double precision.  Waits for the stream.
+ * the device in double precision.  Waits for the stream.  With
+ * ASYNCMESH_FLAG_TRACK_CONSENSUS (where honoured) and at least one step taken it is
+ * the value the last step accumulated on its way; otherwise a read-only pass over
+ * the stage's weights.  The two agree to rounding of the double sum (its order
+ * differs).
  */
 int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *out_host);
 

@@ -97,6 +97,9 @@ struct asyncmesh {
     unsigned int *cursors = nullptr;  // [n_slots][S]
     int *status = nullptr;
     double *scratch = nullptr;        // a few doubles for reductions
+    double *diag = nullptr;           // [S] consensus error accumulated by the last step (tracking kernels)
+    bool tracking = false;
+    uint64_t diag_step = 0;           // the step diag belongs to
 
     int mode = kSync;
     int pipelined = 0;
@@ -437,7 +440,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     if ((cfg->flags & ~(ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_DIRECT_KERNEL |
                         ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE |
                         ASYNCMESH_FLAG_DENSE_RING | ASYNCMESH_FLAG_FP8_EXCHANGE |
-                        ASYNCMESH_FLAG_KEEP_PREVIOUS | ASYNCMESH_FLAG_OWNER_KERNEL)) != 0)
+                        ASYNCMESH_FLAG_KEEP_PREVIOUS | ASYNCMESH_FLAG_OWNER_KERNEL |
+                        ASYNCMESH_FLAG_TRACK_CONSENSUS)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
     if ((cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) && (cfg->flags & ASYNCMESH_FLAG_FP8_EXCHANGE))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: BF16_EXCHANGE and FP8_EXCHANGE exclude each other");
@@ -636,7 +640,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     h->cursors = (unsigned int *)zalloc((size_t)(h->n_slots + 1) * S * sizeof(unsigned int));
     h->status = (int *)zalloc(256);
     h->scratch = (double *)zalloc(256);
-    if (!h->sd_dev || !h->sd_single_dev || !h->cursors || !h->status || !h->scratch)
+    h->diag = (double *)zalloc((size_t)S * sizeof(double));
+    if (!h->sd_dev || !h->sd_single_dev || !h->cursors || !h->status || !h->scratch || !h->diag)
         return bail(ASYNCMESH_ERR_OOM, "out of device memory (tables)");
     std::vector<StageDesc> single(h->sd);
     for (StageDesc &d1 : single) d1.chunk_begin = 0;
@@ -654,6 +659,10 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     // persistent grid: every SM filled to the kernel's occupancy
     h->general = general;
     h->kernel = pick_kernel(R, h->mode, h->pipelined, general, S);
+    if ((cfg->flags & ASYNCMESH_FLAG_TRACK_CONSENSUS) && h->pipelined >= 4 && !general) {
+        h->tracking = true;
+        h->kernel = pick_owner_tracking(R, h->mode, h->pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany, S);
+    }
     int sms = 0, per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
     cudaError_t ke = cudaSuccess;
@@ -759,6 +768,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     P.stages = h->sd_dev;
     P.cursors = h->cursors;
     P.status = h->status;
+    P.diag = h->diag;
     P.S = h->S;
     P.total_chunks = h->total_chunks;
     P.cursor_S = h->S;
@@ -812,6 +822,8 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
         CU_TRY(cudaMemsetAsync(h->cursors + (size_t)P.prod_slot * h->S, 0,
                                h->S * sizeof(unsigned int), h->stream));
 
+    if (h->tracking)   // this step's consensus errors start at zero
+        CU_TRY(cudaMemsetAsync(h->diag, 0, (size_t)h->S * sizeof(double), h->stream));
     if (!stage_ready) {
         h->kernel.fn<<<h->grid, h->kernel.threads, h->kernel.smem, h->stream>>>(P);
         CU_TRY(cudaGetLastError());
@@ -834,6 +846,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
         }
     }
     h->t = t;
+    h->diag_step = t;
     h->mu_product = mu_product;
 
     // roofline numerator (see the header): bytes this step could not avoid
@@ -1069,6 +1082,11 @@ extern "C" int asyncmesh_consensus_error(asyncmesh *h, uint32_t stage, double *o
     int rc = check_status(h, "consensus_error");
     if (rc != ASYNCMESH_OK) return rc;
     const StageDesc &d = h->sd[stage];
+    if (h->tracking && h->t > 0 && h->diag_step == h->t) {   // the last step accumulated it on its way
+        CU_TRY(cudaMemcpyAsync(out_host, h->diag + stage, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+        CU_TRY(cudaStreamSynchronize(h->stream));
+        return ASYNCMESH_OK;
+    }
     CU_TRY(cudaMemsetAsync(h->scratch, 0, sizeof(double), h->stream));
     consensus_for(h->R)<<<grid_for((d.N + 3) / 4, 256), 256, 0, h->stream>>>(d.W, d.stride, d.N, h->scratch);
     CU_TRY(cudaGetLastError());
@@ -1112,7 +1130,7 @@ extern "C" int asyncmesh_kernel_name(const asyncmesh *h, char *buf, size_t cap)
 {
     if (!h || !buf || cap == 0) return fail(ASYNCMESH_ERR_INVALID_ARG, "kernel_name: NULL argument");
     const char *mode = h->mode == kSync ? "sync" : (h->mode == kDense ? "dense" : "compact");
-    const char *form = h->general ? " general" : "";
+    const char *form = h->general ? " general" : (h->tracking ? " tracking" : "");
     switch (h->pipelined) {
     case 0: snprintf(buf, cap, "direct R=%u %s%s", h->R, mode, form); break;
     case 1: snprintf(buf, cap, "pipelined R=%u %s wide%s", h->R, mode, form); break;

@@ -44,5 +44,6 @@ constexpr int kOwnerEntriesFew = 32, kOwnerEntriesMany = 128;
 constexpr int owner_ru(int R) { return (R > 4 && R % 2 == 0) ? 2 : 1; }
 KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S);
 KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S);
+KernelChoice pick_owner_tracking(uint32_t R, int mode, int entries, uint32_t S);   // common form + consensus error
 
 }  // namespace amk

@@ -76,6 +76,7 @@ struct StepParams {
     const StageDesc *stages;     // device [S]
     unsigned int *cursors;       // device [n_slots][S]            (compact only)
     int *status;                 // device status word
+    double *diag;                // device [S]: consensus error per stage, accumulated by the tracking kernels
     const float *G[kMaxStages];  // gradients, [R][stride] each
     uint32_t S, total_chunks;    // stages and warp chunks of THIS launch
     uint32_t cursor_S, s_base;   // stages of the handle and the handle's index of this launch's stage 0:

@@ -227,7 +227,10 @@ __device__ __forceinline__ float div_by_replicas(const StepParams &P, float a)
 }
 
 // MODE kCompact (tau >= 1) or kSync (tau = 0).
-template <int R, int RU, int V, int NST, int E, int MODE, bool GEN>
+// DIAG: the pass also accumulates the consensus error sum_i ||w_i - wbar||^2 of every stage (Section 3.3)
+// from the final weights it holds in registers anyway: no extra memory traffic, fp64 arithmetic per
+// coordinate, one atomicAdd per warp and stage.  A separate set of instantiations.
+template <int R, int RU, int V, int NST, int E, int MODE, bool GEN, bool DIAG = false>
 __global__ void __launch_bounds__(kOwnerThreads, R <= 4 ? kOwnerBlocksPerSM : 2)
 asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
 {
@@ -296,9 +299,22 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
     // flowing while that work runs; this is the very first one.
     const unsigned char *first_slot = advance(std::integral_constant<int, (NST - 1) % UPG>{});
 
+    double diag_acc = 0.0;       // DIAG: this lane's share of the current stage's consensus error
+    uint32_t diag_stage = 0;
+    auto diag_flush = [&]() {
+        for (int d = 16; d > 0; d >>= 1) diag_acc += __shfl_down_sync(kFullMask, diag_acc, d);
+        if (lane == 0 && diag_acc != 0.0) atomicAdd(P.diag + P.s_base + diag_stage, diag_acc);
+        diag_acc = 0.0;
+    };
     uint32_t s = 0;
     for (uint32_t gc = blockIdx.x * wpb + warp; gc < P.total_chunks; gc += n_warps) {
         while (s + 1 < P.S && gc >= sd[s + 1].chunk_begin) ++s;
+        if constexpr (DIAG) {
+            if (s != diag_stage) {   // warp-uniform: the walk has entered another stage
+                diag_flush();
+                diag_stage = s;
+            }
+        }
         const StageDesc &st = sd[s];
         const uint32_t chunk = gc - st.chunk_begin;
         const uint64_t N = st.N, stride = st.stride;
@@ -538,6 +554,22 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                 }
             }
 
+            if constexpr (DIAG) {   // consensus error of the final weights (Section 3.3), in double
+#pragma unroll
+                for (int j = 0; j < NB; ++j) {
+                    if (mu0 + (uint64_t)(j >> 2) * 128 + (j & 3) < N) {
+                        double mean = 0.0;
+#pragma unroll
+                        for (int i = 0; i < R; ++i) mean += (double)wn[i][j];
+                        mean /= (double)R;
+#pragma unroll
+                        for (int i = 0; i < R; ++i) {
+                            const double e = (double)wn[i][j] - mean;
+                            diag_acc += e * e;
+                        }
+                    }
+                }
+            }
             // ---- the one store of w and of the look-ahead (Section 2.2) ----------------
 #pragma unroll
             for (int h = 0; h < V; ++h) {
@@ -561,6 +593,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
             }
         }
     }
+    if constexpr (DIAG) diag_flush();
     cp_async_wait<0>();
 }
 

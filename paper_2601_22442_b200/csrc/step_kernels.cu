@@ -1,12 +1,12 @@
-// Instantiations of the step kernels.  Compiled nine times, -DAM_PART=0..8:
+// Instantiations of the step kernels.  Compiled ten times, -DAM_PART=0..9:
 // 0 direct kernel R = 1..8; 1 direct kernel R = 9..16, common form; 2 the same,
 // general form; 3 / 4 pipelined kernel R = 1..8, common / general form; 5 / 6
-// pipelined kernel R = 9..16, common / general form; 7 / 8 owner kernel R = 1..8,
-// common / general form.
+// pipelined kernel R = 9..16, common / general form; 7 / 8 / 9 owner kernel R = 1..8,
+// common / general / consensus-tracking form.
 #include "kernel_table.cuh"
 
 #ifndef AM_PART
-#error "compile with -DAM_PART=0..8"
+#error "compile with -DAM_PART=0..9"
 #endif
 
 namespace amk {
@@ -70,12 +70,13 @@ KernelChoice pick_direct_many_general(uint32_t R, int mode)
 #elif AM_PART >= 7   // owner kernel
 
 constexpr bool kGeneral = (AM_PART == 8);
+constexpr bool kTracking = (AM_PART == 9);   // the common form that also accumulates the consensus error
 
 template <int R, int E, int MODE>
 static KernelChoice owner_as(uint32_t S)
 {
     KernelChoice c;
-    c.fn = asyncmesh_step_kernel_owner<R, owner_ru(R), kOwnerV, owner_stages(MODE), E, MODE, kGeneral>;
+    c.fn = asyncmesh_step_kernel_owner<R, owner_ru(R), kOwnerV, owner_stages(MODE), E, MODE, kGeneral, kTracking>;
     c.threads = kOwnerThreads;
     c.smem = (size_t)pipe_table_bytes(S) +
              (size_t)(kOwnerThreads / 32) * OwnerCfg<R, owner_ru(R), kOwnerV, E>::warp_bytes(owner_stages(MODE));
@@ -92,8 +93,10 @@ static KernelChoice owner(int mode, int entries, uint32_t S)
 
 #if AM_PART == 7
 KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S)
-#else
+#elif AM_PART == 8
 KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S)
+#else
+KernelChoice pick_owner_tracking(uint32_t R, int mode, int entries, uint32_t S)
 #endif
 {
     switch (R) {

@@ -322,6 +322,33 @@ def test_replicas_starting_apart_and_mean_readback():
         assert abs(ce_o - ce_g) <= 1e-9 * ce_o
 
 
+@pytest.mark.parametrize("R,p,tau,tracked", [(4, 0.1, 1, True), (4, 0.2, 2, True), (3, 0.3, 0, True), (8, 0.3, 0, True),
+                                             (2, 1.0, 0, False), (8, 0.1, 2, False), (4, 1.0, 2, False)])
+def test_consensus_error_tracked_by_the_step_itself(R, p, tau, tracked):
+    # with FLAG_TRACK_CONSENSUS the owner kernel accumulates the consensus error of the final
+    # weights on its way (no second pass); where another kernel runs the flag changes nothing
+    from paper_2601_22442_b200 import binding
+    numel = [6000, 1024 * 2 + 37, 77]
+    o, g = make_pair(R, numel, p, tau, 0.9, same_init=False, flags=binding.FLAG_TRACK_CONSENSUS)
+    assert g.kernel_name().endswith(" tracking") == tracked
+    for s in range(3):
+        assert g.consensus_error(s) > 0           # before any step: the stand-alone pass
+    bufs = None
+    for t in range(1, 2 * tau + 4):
+        bufs = step_both(o, g, t, bufs=bufs)
+        for s in range(3):
+            ce_o, ce_g = o.consensus_error(s), g.consensus_error(s)
+            assert abs(ce_o - ce_g) <= 1e-9 * ce_o, (t, s, ce_o, ce_g)
+    compare(o, g)
+    # through host gradients (one launch per stage) the per-stage sums land in the same places
+    hg = [si.grads_host(0x6AD5, 99, s, R, 0, n) for s, n in enumerate(numel)]
+    o.step(hg)
+    g.step_host(hg)
+    for s in range(3):
+        ce_o, ce_g = o.consensus_error(s), g.consensus_error(s)
+        assert abs(ce_o - ce_g) <= 1e-9 * ce_o, (s, ce_o, ce_g)
+
+
 def test_per_step_schedules():
     o, g = make_pair(2, [4000], 0.3, 1, 0.5)
     bufs = None
