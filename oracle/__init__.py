@@ -56,6 +56,8 @@ def lib() -> ctypes.CDLL:
         L.am_oracle_set_optimizer.argtypes = [vp, u32, dbl]
         L.am_oracle_set_exchange.restype = None
         L.am_oracle_set_exchange.argtypes = [vp, u32]
+        L.am_oracle_set_snapshot_storage.restype = None
+        L.am_oracle_set_snapshot_storage.argtypes = [vp, u32]
         L.am_oracle_set_correction.restype = None
         L.am_oracle_set_correction.argtypes = [vp, u32]
         L.am_oracle_ema_variance.restype = ctypes.c_int
@@ -135,7 +137,8 @@ class Oracle:
                  lookahead_delay: Optional[Sequence[int]] = None,
                  coord_base: Optional[Sequence[int]] = None, avg_interval: int = 1,
                  optimizer: str = "adamw", momentum_decay: float = 4e-3,
-                 exchange: str = "fp32", correction: str = "ema"):
+                 exchange: str = "fp32", correction: str = "ema",
+                 snapshot: str = "own-fp32"):
         self.R, self.S, self.tau = int(R), len(numel), int(tau)
         self.numel = [int(n) for n in numel]
         self.p, self.seed = float(p), int(seed)
@@ -154,6 +157,9 @@ class Oracle:
                                       float(momentum_decay))
         lib().am_oracle_set_exchange(self._h, EXCHANGE[exchange])
         lib().am_oracle_set_correction(self._h, CORRECTION[correction])
+        # "own-fp32": a replica's staleness sample uses its own unrounded snapshot;
+        # "as-exchanged": the snapshot exists only in the exchanged precision
+        lib().am_oracle_set_snapshot_storage(self._h, {"own-fp32": 0, "as-exchanged": 1}[snapshot])
 
     def close(self) -> None:
         if getattr(self, "_h", None):

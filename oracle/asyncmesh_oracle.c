@@ -84,6 +84,8 @@ typedef struct am_oracle {
                              2: rounded to 8-bit floating point (E4M3)                           */
     uint32_t correction;  /* 0: EMA staleness estimate (Eq. "ema"); 1: eager estimate
                              d_i = (w^_i^t - w^_i^{t-tau}) / R (end of Section 3.2)              */
+    uint32_t stored;      /* 0: a replica remembers its own snapshot unrounded; 1: the snapshot
+                             exists only as exchanged (see am_oracle_set_snapshot_storage)       */
     double momentum_decay, mu_product; /* NAdam's momentum schedule and its running product      */
     uint64_t *numel;      /* [S] coordinates held for stage j               */
     uint64_t *coord_base; /* [S] global index of local coordinate 0         */
@@ -278,6 +280,19 @@ void am_oracle_set_correction(am_oracle *o, uint32_t correction)
     if (o) o->correction = correction;
 }
 
+/*
+ * Second reading of the reduced-precision exchange (Section 5.3, paragraph
+ * "Robustness of Sparse Averaging"; Appendix B.2): the paper does not say whether a
+ * replica keeps an unrounded copy of what it sent.  stored = 0 (default): it does,
+ * and its staleness sample w^_i^t - w^_i^{t-tau} uses that copy.  stored = 1: the
+ * snapshot exists only in the exchanged precision, for its owner too, so the sample
+ * is taken against the rounded value and the snapshot memory shrinks with the format.
+ */
+void am_oracle_set_snapshot_storage(am_oracle *o, uint32_t stored)
+{
+    if (o) o->stored = stored;
+}
+
 float am_oracle_exchanged(uint32_t exchange, float x)
 {
     am_oracle tmp;
@@ -357,7 +372,7 @@ int am_oracle_step_ex(am_oracle *o, const float *const *grads, double lambda_t,
                 }
                 wprev[k] = wk;
                 what[k] = wh;
-                Hnow[k] = wh;
+                Hnow[k] = o->stored ? exchanged(o, wh) : wh;
             }
         }
 

@@ -41,8 +41,10 @@ def to_wire(ft, x, wire):
 
 
 def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
-        stage=0, interval=1, wire="fp32", correction="ema"):
-    """grads[t-1][i][mu] for t = 1..T.  Returns a list of per-step records."""
+        stage=0, interval=1, wire="fp32", correction="ema", keeps_own_copy=True):
+    """grads[t-1][i][mu] for t = 1..T.  Returns a list of per-step records.
+    keeps_own_copy: a replica still has the unrounded value it sent tau steps ago for
+    its staleness sample; False: only what went over the wire exists, for everybody."""
     T = len(grads)
     w = [[ft(w0[mu]) for mu in range(N)] for _ in range(R)]
     m = [[ft(0) for _ in range(N)] for _ in range(R)]
@@ -81,7 +83,8 @@ def run(ft, R, N, p, tau, lam, lr, b1, b2, eps, wd, seed, delay, w0, grads,
                     acc = ft(acc + to_wire(ft, old[i][mu], wire))
                 wbar = ft(acc / ft(R))
                 for i in range(R):
-                    stal = ft(what[i][mu] - old[i][mu])
+                    mine = old[i][mu] if keeps_own_copy else to_wire(ft, old[i][mu], wire)
+                    stal = ft(what[i][mu] - mine)
                     if correction == "ema":      # Eq. "ema"
                         d[i][mu] = ft(ft(oml * d[i][mu]) + ft(lamf * stal))
                     else:                        # eager estimate, end of Section 3.2

@@ -545,6 +545,61 @@ def test_bruteforce_trace_with_fp8_exchange(tau):
     assert 1e-4 < diff < 1e-2     # about an E4M3 step (2^-4 relative) of |w| ~ 0.05
 
 
+@pytest.mark.parametrize("wire,lo,hi", [("bf16", 0.0, 1e-3), ("fp8", 1e-4, 2e-2)])
+def test_bruteforce_trace_with_the_snapshot_kept_only_as_exchanged(wire, lo, hi):
+    # second reading of the reduced-precision exchange: the staleness sample is taken
+    # against the rounded snapshot, because nothing else was kept
+    R, N, T, seed, tau = 3, 16, 9, 0x9B, 2
+    w0, grads = rand_setup(R, N, T, seed=35)
+    kw = dict(p=0.5, tau=tau, ema_beta=0.6, seed=seed, lookahead_delay=[1], exchange=wire, **HP)
+    o = oracle.Oracle(R, [N], snapshot="as-exchanged", **kw)
+    first = oracle.Oracle(R, [N], **kw)
+    o.init_params(0, w0); first.init_params(0, w0)
+    args = (R, N, 0.5, tau, 0.6, HP["lr"], HP["beta1"], HP["beta2"], HP["eps"],
+            HP["weight_decay"], seed, 1, w0, grads)
+    tr = bruteforce.run(np.float32, *args, wire=wire, keeps_own_copy=False)
+    for t in range(1, T + 1):
+        o.step([grads[t - 1]]); first.step([grads[t - 1]])
+        for name in ("w", "m", "v", "d", "look"):
+            assert (o.get(0, name).astype(np.float64) == tr[t - 1][name]).all(), (t, name)
+    # the two readings differ in d (it now carries the rounding error of the snapshot) ...
+    diff = np.abs(o.get(0, "d") - first.get(0, "d")).max()
+    assert lo < diff < hi
+    # ... and not at all while the exchange is exact
+    kw["exchange"] = "fp32"
+    a, b = oracle.Oracle(R, [N], snapshot="as-exchanged", **kw), oracle.Oracle(R, [N], **kw)
+    a.init_params(0, w0); b.init_params(0, w0)
+    for t in range(1, T + 1):
+        a.step([grads[t - 1]]); b.step([grads[t - 1]])
+    assert all(np.array_equal(a.get(0, n), b.get(0, n)) for n in ("w", "d", "look"))
+
+
+def test_snapshot_kept_as_exchanged_closed_form_of_one_round():
+    # One replica, p = 1, tau = 1, lambda = 1, no weight decay: at step 2 the average of
+    # one replica is its rounded snapshot q(w^^1), the staleness estimate is
+    # d = w^^2 - q(w^^1), so w^2 = q(w^^1) + (w^^2 - q(w^^1)), all in fp32; under the
+    # first reading d = w^^2 - w^^1 and w^2 = q(w^^1) + (w^^2 - w^^1).
+    N = 64
+    rng = np.random.default_rng(77)
+    w0 = (0.05 * rng.standard_normal(N)).astype(np.float32)
+    g = [(1e-2 * rng.standard_normal((1, N))).astype(np.float32) for _ in range(2)]
+    hp = dict(HP, weight_decay=0.0)
+    for wire in ("bf16", "fp8"):
+        q = lambda x: torch.tensor(x).to({"bf16": torch.bfloat16, "fp8": torch.float8_e4m3fn}[wire]).to(torch.float32).numpy()
+        for snapshot in ("as-exchanged", "own-fp32"):
+            o = oracle.Oracle(1, [N], p=1.0, tau=1, ema_beta=1.0, exchange=wire, snapshot=snapshot, **hp)
+            o.init_params(0, w0)
+            o.step([g[0]])
+            wh1 = o.get(0, "what")[0].copy()
+            o.step([g[1]])
+            wh2 = o.get(0, "what")[0].copy()
+            mine = q(wh1) if snapshot == "as-exchanged" else wh1
+            d = (wh2 - mine).astype(np.float32)
+            assert np.array_equal(o.get(0, "d")[0], d)
+            assert np.array_equal(o.get(0, "w")[0], (q(wh1) + d).astype(np.float32))
+            assert (q(wh1) != wh1).any()
+
+
 # ---- eager staleness estimate (end of Section 3.2) --------------------------------
 
 @pytest.mark.parametrize("p,tau,K", [(1.0, 2, 2), (1.0, 3, 3), (0.5, 2, 1)])
