@@ -85,6 +85,18 @@ extern "C" {
                                           exponent and 3 mantissa bits, nearest even, magnitudes above
                                           448 clamp to 448, no scale factor; the paper does not say
                                           which 8-bit format it used).  Not together with BF16_EXCHANGE */
+#define ASYNCMESH_FLAG_RING_AS_EXCHANGED 1024u /* with BF16_EXCHANGE or FP8_EXCHANGE and tau > 0: a second
+                                                  reading of the reduced-precision exchange (Section 5.3,
+                                                  paragraph "Robustness of Sparse Averaging"; Appendix B.2,
+                                                  which do not say whether a replica keeps an unrounded copy
+                                                  of what it sent).  The snapshot ring stores the values as
+                                                  exchanged, 2 or 1 bytes each, and a replica's staleness
+                                                  sample w^_i^t - w^_i^{t-tau} is taken against that rounded
+                                                  value; d then carries the rounding error of the snapshot.
+                                                  Implies the dense ring (tau slots of R x stride values:
+                                                  half or a quarter of its fp32 size) and the direct kernel;
+                                                  INVALID_ARG without an exchange flag, with tau = 0, or
+                                                  together with SMALL_RING, PIPELINED_KERNEL or OWNER_KERNEL */
 #define ASYNCMESH_FLAG_KEEP_PREVIOUS 128u /* keep w^{t-1}: before each step the weights are copied
                                             aside (one device-to-device copy per stage, 8 bytes per
                                             replica-coordinate of extra traffic, 4 bytes of memory),

@@ -27,6 +27,7 @@ FLAG_FP8_EXCHANGE = 64
 FLAG_KEEP_PREVIOUS = 128
 FLAG_OWNER_KERNEL = 256
 FLAG_TRACK_CONSENSUS = 512
+FLAG_RING_AS_EXCHANGED = 1024
 STATE = {"w": 0, "m": 1, "v": 2, "d": 3, "look": 4}
 
 ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t)

@@ -391,6 +391,7 @@ static KernelChoice pick_kernel(uint32_t R, int mode, int pipelined, bool genera
         return general ? pick_pipelined_few_general(R, pipelined, S) : pick_pipelined_few_common(R, pipelined, S);
     if (pipelined)
         return general ? pick_pipelined_many_general(R, pipelined, S) : pick_pipelined_many_common(R, pipelined, S);
+    if (mode > kDense) return pick_direct_stored(R, mode, general);
     if (R <= 8) return pick_direct_few(R, mode, general);
     return general ? pick_direct_many_general(R, mode) : pick_direct_many_common(R, mode);
 }
@@ -441,8 +442,17 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
                         ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_BF16_EXCHANGE |
                         ASYNCMESH_FLAG_DENSE_RING | ASYNCMESH_FLAG_FP8_EXCHANGE |
                         ASYNCMESH_FLAG_KEEP_PREVIOUS | ASYNCMESH_FLAG_OWNER_KERNEL |
-                        ASYNCMESH_FLAG_TRACK_CONSENSUS)) != 0)
+                        ASYNCMESH_FLAG_TRACK_CONSENSUS | ASYNCMESH_FLAG_RING_AS_EXCHANGED)) != 0)
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: unknown flags");
+    if (cfg->flags & ASYNCMESH_FLAG_RING_AS_EXCHANGED) {
+        if (!(cfg->flags & (ASYNCMESH_FLAG_BF16_EXCHANGE | ASYNCMESH_FLAG_FP8_EXCHANGE)) || cfg->tau == 0)
+            return fail(ASYNCMESH_ERR_INVALID_ARG,
+                        "create: RING_AS_EXCHANGED needs BF16_EXCHANGE or FP8_EXCHANGE and tau > 0");
+        if (cfg->flags & (ASYNCMESH_FLAG_SMALL_RING | ASYNCMESH_FLAG_PIPELINED_KERNEL | ASYNCMESH_FLAG_OWNER_KERNEL))
+            return fail(ASYNCMESH_ERR_INVALID_ARG,
+                        "create: RING_AS_EXCHANGED uses the dense ring and the direct kernel: not together with "
+                        "SMALL_RING, PIPELINED_KERNEL or OWNER_KERNEL");
+    }
     if ((cfg->flags & ASYNCMESH_FLAG_BF16_EXCHANGE) && (cfg->flags & ASYNCMESH_FLAG_FP8_EXCHANGE))
         return fail(ASYNCMESH_ERR_INVALID_ARG, "create: BF16_EXCHANGE and FP8_EXCHANGE exclude each other");
     if (cfg->optimizer > ASYNCMESH_OPT_NADAMW || cfg->correction > ASYNCMESH_CORRECTION_EAGER ||
@@ -535,6 +545,9 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
     h->total_chunks = (uint32_t)chunks;
     if (h->tau == 0) { h->mode = kSync; h->n_slots = 0; }
+    else if (cfg->flags & ASYNCMESH_FLAG_RING_AS_EXCHANGED) {
+        h->mode = h->wire == 1u ? kDenseBf16 : kDenseE4m3; h->n_slots = h->lag;
+    }
     else if ((cfg->flags & ASYNCMESH_FLAG_DENSE_RING) && !(cfg->flags & ASYNCMESH_FLAG_SMALL_RING)) {
         h->mode = kDense; h->n_slots = h->lag;
     }
@@ -570,7 +583,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     // kernel carries that form's optimizer code four times over (once per unit of a
     // group) and loses more to it than the pipelined kernel does (1B layout, NAdamW: 30.1
     // against 24.1 ms per step), so the general form stays with the pipelined kernel.
-    const bool general = h->wire == 2u || h->correction == ASYNCMESH_CORRECTION_EAGER ||
+    // (a ring kept as exchanged converts by its slot format, which is a template parameter: common form)
+    const bool general = (h->wire == 2u && h->mode <= kDense) || h->correction == ASYNCMESH_CORRECTION_EAGER ||
                          h->optimizer == ASYNCMESH_OPT_NADAMW;
     const bool owner_asked = (cfg->flags & ASYNCMESH_FLAG_OWNER_KERNEL) != 0;
     const bool owner_default =
@@ -578,7 +592,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         (h->mode == kCompact || (h->mode == kSync && cfg->p <= 0.8));
     // (five to eight replicas: for tau = 0 only; 350M layout, p = 0.05: 14.15 against 15.09 ms, while with
     // the ring the pipelined kernel is as fast at p = 0.05 and faster at p = 0.01 and 0.25)
-    if ((R <= 4 || (R <= 8 && h->mode == kSync)) && h->mode != kDense && (owner_asked || owner_default)) {
+    if ((R <= 4 || (R <= 8 && h->mode == kSync)) && !is_dense(h->mode) && (owner_asked || owner_default)) {
         const double mean = 128.0 * kOwnerV * cfg->p, sd = std::sqrt(mean * (1.0 - cfg->p));
         h->pipelined = h->mode == kSync ? 6 : (mean + 4.0 * sd <= (double)kOwnerEntriesFew ? 4 : 5);
     }
@@ -627,11 +641,11 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
                 d.bitmap = (uint32_t *)zalloc((size_t)h->n_slots * d.n_chunks * 32 * sizeof(uint32_t));
                 if (!d.bitmap) return bail(ASYNCMESH_ERR_OOM, "out of device memory (subset masks)");
             }
-        } else if (h->mode == kDense) {
-            d.slot_floats = h->stride[s] * R;
+        } else if (is_dense(h->mode)) {
+            d.slot_floats = h->stride[s] * R;   // values per slot, ring_value_bytes(mode) each
         }
         if (h->mode != kSync) {
-            d.ring = (float *)zalloc((size_t)h->n_slots * d.slot_floats * sizeof(float));
+            d.ring = (float *)zalloc((size_t)h->n_slots * d.slot_floats * (size_t)ring_value_bytes(h->mode));
             if (!d.ring) return bail(ASYNCMESH_ERR_OOM, "out of device memory (snapshot ring)");
         }
     }
@@ -783,7 +797,7 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     if (h->mode == kCompact) {
         P.prod_slot = (uint32_t)(r % (h->lag + 1));
         P.cons_slot = (uint32_t)((r - h->lag) % (h->lag + 1));   // unused while t <= tau
-    } else if (h->mode == kDense) {
+    } else if (is_dense(h->mode)) {
         P.prod_slot = P.cons_slot = (uint32_t)(r % h->lag);
     }
     P.rule = h->rule;
@@ -853,7 +867,9 @@ static int launch_step(asyncmesh *h, const float *const *grads, double ema_beta_
     double bytes = 0.0;
     for (uint32_t s = 0; s < h->S; ++s) {
         double per = 28.0 + (h->delay[s] ? 4.0 : 0.0);
-        if (h->mode != kSync && round) per += 4.0 * h->p + (P.consume ? 12.0 * h->p : 0.0);
+        // snapshot written, and on arrival read again with d read and written
+        const double rb = h->mode == kSync ? 0.0 : (double)ring_value_bytes(h->mode);
+        if (h->mode != kSync && round) per += rb * h->p + (P.consume ? (rb + 8.0) * h->p : 0.0);
         bytes += per * (double)h->R * (double)h->numel[s];
     }
     h->last_bytes = (uint64_t)bytes;
@@ -1009,7 +1025,7 @@ extern "C" int asyncmesh_read_state_range(asyncmesh *h, uint32_t stage, int whic
     case ASYNCMESH_STATE_M: row = d.M; break;
     case ASYNCMESH_STATE_V: row = d.V; break;
     case ASYNCMESH_STATE_LOOK: row = d.LOOK; break;
-    case ASYNCMESH_STATE_D: if (h->mode == kDense) row = d.D; break;   // replica-major there
+    case ASYNCMESH_STATE_D: if (is_dense(h->mode)) row = d.D; break;   // replica-major there
     default: return fail(ASYNCMESH_ERR_INVALID_ARG, "read_state: unknown selector %d", which);
     }
     if (row) {
@@ -1106,7 +1122,7 @@ extern "C" int asyncmesh_ema_variance(asyncmesh *h, uint32_t stage, double *mean
     const StageDesc &d = h->sd[stage];
     // d is coordinate-major [stride][R] except with the dense ring ([R][stride])
     CU_TRY(cudaMemsetAsync(h->scratch, 0, 2 * sizeof(double), h->stream));
-    if (h->mode == kDense)
+    if (is_dense(h->mode))
         spread_for<1>(h->R)<<<grid_for((d.N + 3) / 4, 256), 256, 0, h->stream>>>(d.D, d.stride, d.N, h->scratch);
     else
         spread_for<0>(h->R)<<<grid_for(d.N, 256), 256, 0, h->stream>>>(d.D, d.stride, d.N, h->scratch);
@@ -1129,7 +1145,8 @@ extern "C" int asyncmesh_step_count(const asyncmesh *h, uint64_t *t)
 extern "C" int asyncmesh_kernel_name(const asyncmesh *h, char *buf, size_t cap)
 {
     if (!h || !buf || cap == 0) return fail(ASYNCMESH_ERR_INVALID_ARG, "kernel_name: NULL argument");
-    const char *mode = h->mode == kSync ? "sync" : (h->mode == kDense ? "dense" : "compact");
+    const char *mode = h->mode == kSync ? "sync" : h->mode == kDense ? "dense" : h->mode == kDenseBf16 ? "dense-bf16"
+                       : h->mode == kDenseE4m3 ? "dense-e4m3" : "compact";
     const char *form = h->general ? " general" : (h->tracking ? " tracking" : "");
     switch (h->pipelined) {
     case 0: snprintf(buf, cap, "direct R=%u %s%s", h->R, mode, form); break;

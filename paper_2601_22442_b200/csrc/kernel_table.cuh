@@ -1,6 +1,6 @@
 // Which step kernel serves which configuration.  The instantiations (every
 // replica count 1..16, three ring modes, two pipelined shapes) take minutes to
-// compile in one translation unit, so step_kernels.cu is compiled in seven parts
+// compile in one translation unit, so step_kernels.cu is compiled in eleven parts
 // side by side; this header is what the host code sees of them.
 #pragma once
 #include "step_kernel_pipelined.cuh"
@@ -22,6 +22,7 @@ struct KernelChoice {
 KernelChoice pick_direct_few(uint32_t R, int mode, bool general);    // R = 1..8
 KernelChoice pick_direct_many_common(uint32_t R, int mode);          // R = 9..16
 KernelChoice pick_direct_many_general(uint32_t R, int mode);
+KernelChoice pick_direct_stored(uint32_t R, int mode, bool general);  // R = 1..16; kDenseBf16 or kDenseE4m3
 // Pipelined kernel.  shape: 1 wide, 2 narrow (both compact ring), 3 narrow synchronous.
 KernelChoice pick_pipelined_few_common(uint32_t R, int shape, uint32_t S);     // R = 1..8
 KernelChoice pick_pipelined_few_general(uint32_t R, int shape, uint32_t S);

@@ -51,7 +51,11 @@ constexpr uint32_t kInvalidBase = 0xFFFFFFFFu;
 constexpr unsigned kFullMask = 0xFFFFFFFFu;
 constexpr int kMaxStages = 64;
 
-enum RingMode : int { kSync = 0, kCompact = 1, kDense = 2 };
+// kDenseBf16 / kDenseE4m3: the dense ring holding the snapshot only as exchanged
+// (2 or 1 bytes per value; the staleness sample is taken against that rounded value)
+enum RingMode : int { kSync = 0, kCompact = 1, kDense = 2, kDenseBf16 = 3, kDenseE4m3 = 4 };
+constexpr bool is_dense(int mode) { return mode >= kDense; }
+constexpr int ring_value_bytes(int mode) { return mode == kDenseBf16 ? 2 : (mode == kDenseE4m3 ? 1 : 4); }
 
 constexpr int kStatusRingOverflow = 1;
 
@@ -227,6 +231,49 @@ __device__ __forceinline__ void adamw_group(const StepParams &P, const float (&w
     }
 }
 
+// Four consecutive values of a dense ring slot, `off` values from the start of the ring
+// (a multiple of 4), in the slot's own format; widening bfloat16 or E4M3 to fp32 is exact.
+template <int MODE>
+__device__ __forceinline__ float4 ring_load4(const float *ring, uint64_t off)
+{
+    if constexpr (MODE == kDenseBf16) {
+        const uint2 u = *reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(ring) + off);
+        return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u),
+                           __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u));
+    } else if constexpr (MODE == kDenseE4m3) {
+        const uint32_t u = *reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint8_t *>(ring) + off);
+        float x[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            x[c] = __half2float(__half(__nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)((u >> (8 * c)) & 0xFFu), __NV_E4M3)));
+        return make_float4(x[0], x[1], x[2], x[3]);
+    } else {
+        return *reinterpret_cast<const float4 *>(ring + off);
+    }
+}
+
+// ... and the snapshot of four local iterates into it: rounded to nearest even (E4M3
+// clamps at its largest finite value 448) where the slot is narrower than fp32.
+template <int MODE>
+__device__ __forceinline__ void ring_store4(float *ring, uint64_t off, const float (&x)[4])
+{
+    if constexpr (MODE == kDenseBf16) {
+        uint32_t h[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) h[c] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x[c]));
+        __stcs(reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(ring) + off),
+               make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16)));
+    } else if constexpr (MODE == kDenseE4m3) {
+        uint32_t u = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            u |= (uint32_t)__nv_cvt_float_to_fp8(x[c], __NV_SATFINITE, __NV_E4M3) << (8 * c);
+        __stcs(reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(ring) + off), u);
+    } else {
+        st_stream(ring + off, x);
+    }
+}
+
 template <int R>
 __device__ __forceinline__ void load_replicas(const float *p, float (&x)[R])
 {
@@ -269,6 +316,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
     const uint64_t N = st.N, stride = st.stride;
     const uint64_t c0 = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
     const bool consume = (MODE != kSync) && (P.consume != 0u);
+    constexpr bool kStored = MODE > kDense;   // the slot holds values already rounded for the exchange
 
     // ---- membership of this lane's 32 coordinates in S^t and S^{t-tau} --------
     uint32_t pmask = 0, cmask = 0;   // bit 4k+j: coordinate c0 + 128k + j
@@ -312,8 +360,10 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
             cexcl = warp_exclusive_sum(__popc(cmask), lane, ctotal);
         }
     }
-    const float *ring_cons = st.ring + (uint64_t)P.cons_slot * st.slot_floats;
-    float *ring_prod = st.ring + (uint64_t)P.prod_slot * st.slot_floats;
+    const uint64_t cons_off = (uint64_t)P.cons_slot * st.slot_floats;   // in ring values
+    const uint64_t prod_off = (uint64_t)P.prod_slot * st.slot_floats;
+    const float *ring_cons = st.ring + cons_off;
+    float *ring_prod = st.ring + prod_off;
     const float delta = st.delta;
     const bool has_look = st.delta != 0.0f;
 
@@ -324,7 +374,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
         const uint32_t pm = (pmask >> (4 * k)) & 0xFu;
         const uint32_t cm = (cmask >> (4 * k)) & 0xFu;
 
-        if constexpr (MODE == kDense) {
+        if constexpr (MODE >= kDense) {
             // Large subsets: the ring slot and d are replica-major like w, m, v, so the
             // sparse quantities stream as float4 too.  A lane owns its four coordinates
             // in every replica row, reads a ring position before it overwrites it, and
@@ -338,7 +388,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
 #pragma unroll
             for (int i = 0; i < R; ++i) {
                 r4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (cm) r4[i] = *reinterpret_cast<const float4 *>(ring_cons + (uint64_t)i * stride + mu);
+                if (cm) r4[i] = ring_load4<MODE>(st.ring, cons_off + (uint64_t)i * stride + mu);
             }
             float abar[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -360,8 +410,10 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                     for (int i = 0; i < R; ++i) {
                         const float r[4] = {r4[i].x, r4[i].y, r4[i].z, r4[i].w};
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            a[c] = (i == 0) ? on_wire<GEN>(P, r[c]) : __fadd_rn(a[c], on_wire<GEN>(P, r[c]));
+                        for (int c = 0; c < 4; ++c) {
+                            const float sent = kStored ? r[c] : on_wire<GEN>(P, r[c]);
+                            a[c] = (i == 0) ? sent : __fadd_rn(a[c], sent);
+                        }
                     }
 #pragma unroll
                     for (int c = 0; c < 4; ++c) abar[c] = __fdiv_rn(a[c], P.Rf);
@@ -393,7 +445,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
                         }
                         st_stream(st.D + off, dd);
                     }
-                    if (pm) st_stream(ring_prod + off, wh);   // snapshot of the local iterate on S^t
+                    if (pm) ring_store4<MODE>(st.ring, prod_off + off, wh);   // snapshot of the local iterate on S^t
                     st_stream(st.W + off, wn);
                     if (has_look) {
                         float lk[4];
@@ -416,9 +468,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     if ((cm >> j) & 1u) {
-                        const uint64_t idx = (MODE == kDense)
-                            ? (mu + j)
-                            : (uint64_t)(cbase + cexcl + below + __popc(cm & ((1u << j) - 1u)));
+                        const uint64_t idx = (uint64_t)(cbase + cexcl + below + __popc(cm & ((1u << j) - 1u)));
                         ce[j] = idx * R;
                         float old[R];
                         load_replicas<R>(ring_cons + ce[j], old);
@@ -434,9 +484,7 @@ __device__ __forceinline__ void process_chunk(const StepParams &P, const StageDe
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     if ((pm >> j) & 1u) {
-                        const uint64_t idx = (MODE == kDense)
-                            ? (mu + j)
-                            : (uint64_t)(pbase + pexcl + below + __popc(pm & ((1u << j) - 1u)));
+                        const uint64_t idx = (uint64_t)(pbase + pexcl + below + __popc(pm & ((1u << j) - 1u)));
                         pe[j] = idx * R;
                     }
                 }

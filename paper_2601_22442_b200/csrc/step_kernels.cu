@@ -1,17 +1,54 @@
-// Instantiations of the step kernels.  Compiled ten times, -DAM_PART=0..9:
+// Instantiations of the step kernels.  Compiled eleven times, -DAM_PART=0..10:
 // 0 direct kernel R = 1..8; 1 direct kernel R = 9..16, common form; 2 the same,
 // general form; 3 / 4 pipelined kernel R = 1..8, common / general form; 5 / 6
 // pipelined kernel R = 9..16, common / general form; 7 / 8 / 9 owner kernel R = 1..8,
-// common / general / consensus-tracking form.
+// common / general / consensus-tracking form; 10 direct kernel with the dense ring kept as
+// exchanged (bfloat16 / E4M3 slots), R = 1..16, both forms.
 #include "kernel_table.cuh"
 
 #ifndef AM_PART
-#error "compile with -DAM_PART=0..9"
+#error "compile with -DAM_PART=0..10"
 #endif
 
 namespace amk {
 
-#if AM_PART < 3
+#if AM_PART == 10   // direct kernel, ring slots in the exchanged precision
+
+template <int R>
+static KernelChoice stored(int mode, bool general)
+{
+    KernelChoice c;
+    if (mode == kDenseBf16)
+        c.fn = general ? asyncmesh_step_kernel<R, kDenseBf16, true> : asyncmesh_step_kernel<R, kDenseBf16, false>;
+    else if (mode == kDenseE4m3)
+        c.fn = general ? asyncmesh_step_kernel<R, kDenseE4m3, true> : asyncmesh_step_kernel<R, kDenseE4m3, false>;
+    return c;
+}
+
+KernelChoice pick_direct_stored(uint32_t R, int mode, bool general)
+{
+    switch (R) {
+    case 1: return stored<1>(mode, general);
+    case 2: return stored<2>(mode, general);
+    case 3: return stored<3>(mode, general);
+    case 4: return stored<4>(mode, general);
+    case 5: return stored<5>(mode, general);
+    case 6: return stored<6>(mode, general);
+    case 7: return stored<7>(mode, general);
+    case 8: return stored<8>(mode, general);
+    case 9: return stored<9>(mode, general);
+    case 10: return stored<10>(mode, general);
+    case 11: return stored<11>(mode, general);
+    case 12: return stored<12>(mode, general);
+    case 13: return stored<13>(mode, general);
+    case 14: return stored<14>(mode, general);
+    case 15: return stored<15>(mode, general);
+    case 16: return stored<16>(mode, general);
+    default: return KernelChoice();
+    }
+}
+
+#elif AM_PART < 3
 
 template <int R, bool GEN>
 static KernelChoice direct_as(int mode)

@@ -65,7 +65,9 @@ def _cfg(**over):
     (dict(p=-0.1), "p ="), (dict(p=1.5), "p ="), (dict(p=float("nan")), "p ="),
     (dict(tau=65), "tau"), (dict(ema_beta=1.01), "ema_beta"), (dict(lr=0.0), "lr"),
     (dict(eps=0.0), "eps"), (dict(beta1=1.0), "betas"), (dict(tau=3, avg_interval=2), "avg_interval"),
-    (dict(avg_interval=-1), "avg_interval"), (dict(optimizer=2), "optimizer"), (dict(flags=8), "flags"), (dict(flags=1024), "flags"),
+    (dict(avg_interval=-1), "avg_interval"), (dict(optimizer=2), "optimizer"), (dict(flags=8), "flags"), (dict(flags=2048), "flags"),
+    (dict(flags=1024), "RING_AS_EXCHANGED"), (dict(flags=1024 | 16, tau=0), "RING_AS_EXCHANGED"),
+    (dict(flags=1024 | 64 | 4), "RING_AS_EXCHANGED"), (dict(flags=1024 | 16 | 256), "RING_AS_EXCHANGED"),
     (dict(flags=16 | 64), "exclude"), (dict(correction=2), "correction"),
     (dict(coord_base=(ctypes.c_uint64 * 1)(6)), "coord_base"),
     (dict(coord_base=(ctypes.c_uint64 * 1)(2 ** 32 - 4)), "coord_base"),

@@ -70,10 +70,12 @@ def same_bits(a, b, what):
                            % (bad.size, bad[0], a[~na][bad[0]], b[~nb][bad[0]]))
 
 
-def run(R, n, p, tau, flags, exchange="fp32", steps=7, seed=0, optimizer="adamw"):
+def run(R, n, p, tau, flags, exchange="fp32", steps=7, seed=0, optimizer="adamw", snapshot="own-fp32"):
     numel = [n, n // 2 + 3]       # two stages: look-ahead delays 1 and 0
     xflag = {"fp32": 0, "bf16": 16, "fp8": 64}[exchange]
-    o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=0.9, seed=11, exchange=exchange, optimizer=optimizer, **HP)
+    o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=0.9, seed=11, exchange=exchange, optimizer=optimizer,
+                      snapshot=snapshot, **HP)
+    flags |= {"own-fp32": 0, "as-exchanged": 1024}[snapshot]
     g = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=0.9, seed=11, flags=flags | xflag, optimizer=optimizer, **HP)
     inputs = [build_inputs(R, m, steps, seed + s) for s, m in enumerate(numel)]
     for s in range(2):
@@ -131,6 +133,14 @@ def test_edge_values_with_the_8_bit_exchange(kernel, R):
     # weights beyond the largest E4M3 value (448) clamp in the exchange; NaN stays NaN
     run(R, 2 * 1024 + 7, 0.3, 2, flags_of(kernel), exchange="fp8")
     run(R, 1024 + 7, 0.3, 0, flags_of(kernel) & ~32, exchange="bf16", steps=4)
+
+
+@pytest.mark.parametrize("exchange", ["bf16", "fp8"])
+@pytest.mark.parametrize("R", [1, 4, 8])
+def test_edge_values_with_the_ring_kept_as_exchanged(exchange, R):
+    # infinities, NaN, subnormals and values beyond 448 pass through the 2- and 1-byte ring slots
+    run(R, 2 * 1024 + 7, 0.5, 2, 0, exchange=exchange, snapshot="as-exchanged")
+    run(R, 1024 + 7, 1.0, 1, 0, exchange=exchange, snapshot="as-exchanged", steps=4)
 
 
 def test_edge_values_nadamw():

@@ -154,3 +154,12 @@ def test_general_forms():
     run(4, [4099, 77], 0.3, 2, flags=16)
     run(4, [4099, 77], 0.3, 2, optimizer="nadamw")
     run(8, [4099, 77], 0.3, 2, correction="eager")
+
+
+def test_ring_kept_as_exchanged():
+    # (delays chosen so that the ring block is not of a state array's size)
+    run(4, RAGGED, 0.4, 1, flags=16 | 1024)
+    run(8, RAGGED, 1.0, 3, flags=16 | 1024)
+    run(3, RAGGED, 0.4, 2, flags=64 | 1024)
+    run(16, [4099, 130], 1.0, 1, flags=64 | 1024)
+    run(5, [4099, 130], 0.7, 3, flags=64 | 1024, optimizer="nadamw")

@@ -27,11 +27,12 @@ def am():
 
 def make_pair(R, numel, p, tau, lam, delays=None, seed=0x5EED, hp=HP, same_init=True,
               init_seed=0x1217, flags=0, avg_interval=1, optimizer="adamw", exchange="fp32",
-              correction="ema"):
+              correction="ema", snapshot="own-fp32"):
     flags |= {"fp32": 0, "bf16": 16, "fp8": 64}[exchange]
+    flags |= {"own-fp32": 0, "as-exchanged": 1024}[snapshot]
     o = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
                       lookahead_delay=delays, avg_interval=avg_interval, optimizer=optimizer,
-                      exchange=exchange, correction=correction, **hp)
+                      exchange=exchange, correction=correction, snapshot=snapshot, **hp)
     g = am().AsyncMesh(R, numel, p=p, tau=tau, ema_beta=lam, seed=seed,
                        lookahead_delay=delays, flags=flags, avg_interval=avg_interval,
                        optimizer=optimizer, correction=correction, **hp)
@@ -240,6 +241,63 @@ def test_fp8_exchange(tau, p):
     for t in range(1, 3 * tau + 6):
         ref.step([si.grads_host(0x6AD5, t, s, 4, 0, n) for s, n in enumerate([6000, 1024 + 9])])
     assert np.abs(ref.get(0, "w") - g.get(0, "w")).max() > 0    # nor is it the bfloat16 exchange
+
+
+@pytest.mark.parametrize("exchange", ["bf16", "fp8"])
+@pytest.mark.parametrize("R,tau,p,K", [(4, 2, 1.0, 1), (3, 1, 0.3, 1), (8, 3, 0.6, 1), (1, 2, 1.0, 1),
+                                       (2, 4, 0.9, 2), (12, 2, 0.5, 1), (16, 1, 1.0, 1)])
+def test_ring_kept_as_exchanged(exchange, R, tau, p, K):
+    # second reading of the reduced-precision exchange: the ring holds 2- or 1-byte values and
+    # the staleness sample is taken against them
+    numel = [6000, 1024 + 9, 77]
+    o, g = run_case(R, numel, p, tau, 0.9, steps=3 * tau + 5, exchange=exchange, snapshot="as-exchanged",
+                    avg_interval=K)
+    assert g.kernel_name() == "direct R=%d dense-%s" % (R, {"bf16": "bf16", "fp8": "e4m3"}[exchange])
+    # it is not the first reading: d differs
+    first = oracle.Oracle(R, numel, p=p, tau=tau, ema_beta=0.9, exchange=exchange, avg_interval=K, **HP)
+    for s, n in enumerate(numel):
+        first.init_params(s, si.init_weights_host(0x1217, s, 0, n))
+    for t in range(1, 3 * tau + 6):
+        first.step([si.grads_host(0x6AD5, t, s, R, 0, n) for s, n in enumerate(numel)])
+    assert np.abs(first.get(0, "d") - g.get(0, "d")).max() > 0
+
+
+def test_ring_kept_as_exchanged_general_form_and_schedules():
+    run_case(4, [6000, 77], 0.5, 2, 0.9, steps=9, exchange="fp8", snapshot="as-exchanged", optimizer="nadamw")
+    run_case(8, [6000, 77], 1.0, 2, 0.9, steps=9, exchange="bf16", snapshot="as-exchanged", correction="eager")
+    o, g = make_pair(4, [5000], 0.7, 2, 0.9, exchange="bf16", snapshot="as-exchanged", same_init=False)
+    bufs = None
+    for t in range(1, 9):
+        bufs = step_both(o, g, t, bufs=bufs, ema_beta_t=0.9 * 0.8 ** t, lr_t=3e-4 * (1 - t / 20))
+    g.status()
+    compare(o, g)
+
+
+def test_ring_kept_as_exchanged_takes_half_or_a_quarter_of_the_ring_memory():
+    from paper_2601_22442_b200 import binding
+    from paper_2601_22442_b200.binding import TorchAllocator
+
+    class Counting(TorchAllocator):
+        def __init__(self):
+            super().__init__(0)
+            self.sizes = []
+
+        def _alloc(self, ctx, nbytes):
+            self.sizes.append(int(nbytes))
+            return super()._alloc(ctx, nbytes)
+
+    R, N, tau = 4, 1 << 20, 6
+    ring = {}
+    for name, flags in (("fp32", binding.FLAG_DENSE_RING), ("bf16", 16 | 1024), ("e4m3", 64 | 1024)):
+        a = Counting()
+        g = am().AsyncMesh(R, [N], p=1.0, tau=tau, ema_beta=0.9, flags=flags, allocator=a, **HP)
+        g.destroy()
+        # the ring is one block of tau slots of R x N values; nothing else is larger than a state array
+        want = tau * R * N * {"fp32": 4, "bf16": 2, "e4m3": 1}[name]
+        assert a.sizes.count(want) == 1, (name, sorted(a.sizes)[-8:])
+        assert all(n <= R * N * 4 for n in a.sizes if n != want)
+        ring[name] = sum(a.sizes)
+    assert ring["fp32"] - ring["bf16"] == tau * R * N * 2 and ring["fp32"] - ring["e4m3"] == tau * R * N * 3
 
 
 def test_fp8_conversion_on_the_device_covers_the_whole_format():
