@@ -25,9 +25,9 @@ NVCC_FLAGS = [
 ]
 
 # translation units: the C ABI with its small kernels, and the step-kernel
-# instantiations in eleven parts that compile side by side
+# instantiations in twelve parts that compile side by side
 UNITS = [("asyncmesh", "asyncmesh.cu", []),
-         *[("step_kernels_%d" % k, "step_kernels.cu", ["-DAM_PART=%d" % k]) for k in range(11)]]
+         *[("step_kernels_%d" % k, "step_kernels.cu", ["-DAM_PART=%d" % k]) for k in range(12)]]
 
 
 def nvcc() -> str:

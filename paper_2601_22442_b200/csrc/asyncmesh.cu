@@ -104,6 +104,7 @@ struct asyncmesh {
     int mode = kSync;
     int pipelined = 0;
     bool general = false;             // the kernels' general form (E4M3 exchange, eager estimate, NAdamW)
+    bool nadam_form = false;          // the owner kernel's common form with NAdamW fixed at compile time
     KernelChoice kernel;
     uint32_t n_slots = 0;
     uint32_t total_chunks = 0;
@@ -586,9 +587,17 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     // (a ring kept as exchanged converts by its slot format, which is a template parameter: common form)
     const bool general = (h->wire == 2u && h->mode <= kDense) || h->correction == ASYNCMESH_CORRECTION_EAGER ||
                          h->optimizer == ASYNCMESH_OPT_NADAMW;
+    // NAdamW alone (the optimizer of the paper's asynchronous-pipeline runs) has an owner form of its
+    // own, with the optimizer fixed at compile time.  1B layout, ms per step, that form against the
+    // pipelined kernel's general form: tau = 0 19.56 / 21.34, so it is the default there; with the ring
+    // 26.2 / 24.3 at p = 0.05 and 32.1 / 30.0 at p = 0.25 (the second division costs the owner kernel,
+    // which has no registers to spare at three blocks per SM, more than it costs the pipelined one):
+    // there only on ASYNCMESH_FLAG_OWNER_KERNEL, where it replaces the general form's 30.1.
+    const bool nadam_only = h->optimizer == ASYNCMESH_OPT_NADAMW && h->wire != 2u &&
+                            h->correction != ASYNCMESH_CORRECTION_EAGER;
     const bool owner_asked = (cfg->flags & ASYNCMESH_FLAG_OWNER_KERNEL) != 0;
     const bool owner_default =
-        !general && !(cfg->flags & (ASYNCMESH_FLAG_DIRECT_KERNEL | ASYNCMESH_FLAG_PIPELINED_KERNEL)) &&
+        (!general || (nadam_only && h->mode == kSync)) && !(cfg->flags & (ASYNCMESH_FLAG_DIRECT_KERNEL | ASYNCMESH_FLAG_PIPELINED_KERNEL)) &&
         (h->mode == kCompact || (h->mode == kSync && cfg->p <= 0.8));
     // (five to eight replicas: for tau = 0 only; 350M layout, p = 0.05: 14.15 against 15.09 ms, while with
     // the ring the pipelined kernel is as fast at p = 0.05 and faster at p = 0.01 and 0.25)
@@ -671,8 +680,11 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
 
     // persistent grid: every SM filled to the kernel's occupancy
-    h->general = general;
-    h->kernel = pick_kernel(R, h->mode, h->pipelined, general, S);
+    h->nadam_form = h->pipelined >= 4 && nadam_only;
+    h->general = general && !h->nadam_form;
+    h->kernel = h->nadam_form
+        ? pick_owner_nadamw(R, h->mode, h->pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany, S)
+        : pick_kernel(R, h->mode, h->pipelined, general, S);
     if ((cfg->flags & ASYNCMESH_FLAG_TRACK_CONSENSUS) && h->pipelined >= 4 && !general) {
         h->tracking = true;
         h->kernel = pick_owner_tracking(R, h->mode, h->pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany, S);
@@ -1147,7 +1159,7 @@ extern "C" int asyncmesh_kernel_name(const asyncmesh *h, char *buf, size_t cap)
     if (!h || !buf || cap == 0) return fail(ASYNCMESH_ERR_INVALID_ARG, "kernel_name: NULL argument");
     const char *mode = h->mode == kSync ? "sync" : h->mode == kDense ? "dense" : h->mode == kDenseBf16 ? "dense-bf16"
                        : h->mode == kDenseE4m3 ? "dense-e4m3" : "compact";
-    const char *form = h->general ? " general" : (h->tracking ? " tracking" : "");
+    const char *form = h->general ? " general" : h->tracking ? " tracking" : h->nadam_form ? " nadamw" : "";
     switch (h->pipelined) {
     case 0: snprintf(buf, cap, "direct R=%u %s%s", h->R, mode, form); break;
     case 1: snprintf(buf, cap, "pipelined R=%u %s wide%s", h->R, mode, form); break;

@@ -1,6 +1,6 @@
 // Which step kernel serves which configuration.  The instantiations (every
 // replica count 1..16, three ring modes, two pipelined shapes) take minutes to
-// compile in one translation unit, so step_kernels.cu is compiled in eleven parts
+// compile in one translation unit, so step_kernels.cu is compiled in twelve parts
 // side by side; this header is what the host code sees of them.
 #pragma once
 #include "step_kernel_pipelined.cuh"
@@ -46,5 +46,6 @@ constexpr int owner_ru(int R) { return (R > 4 && R % 2 == 0) ? 2 : 1; }
 KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S);
 KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S);
 KernelChoice pick_owner_tracking(uint32_t R, int mode, int entries, uint32_t S);   // common form + consensus error
+KernelChoice pick_owner_nadamw(uint32_t R, int mode, int entries, uint32_t S);     // common form, NAdamW for AdamW
 
 }  // namespace amk

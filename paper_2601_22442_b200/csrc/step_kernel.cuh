@@ -158,7 +158,42 @@ static __device__ __noinline__ float adam_quotient_anyrange(float mh, float vh, 
 // when every operand of the group lies in their range (one test per group; eps is
 // tested by the host: P.eps_inrange), else the toolkit's routines: the same bits
 // either way.
-template <bool GEN, int NC>
+// NAdamW (Appendix B.1) from the moments of this step: gradient part and (uncorrected)
+// momentum part over the same denominator, weighted by the momentum schedule's cg and cm.
+template <int NC>
+__device__ __forceinline__ void nadamw_finish(const StepParams &P, const float (&w)[NC], const float (&g)[NC],
+                                              const float (&m)[NC], const float (&vh)[NC], float (&what)[NC])
+{
+    float vlo = vh[0], vhi = vh[0], alo = fminf(fabsf(g[0]), fabsf(m[0])),
+          ahi = fmaxf(fabsf(g[0]), fabsf(m[0]));
+#pragma unroll
+    for (int c = 1; c < NC; ++c) {
+        vlo = fminf(vlo, vh[c]);
+        vhi = fmaxf(vhi, vh[c]);
+        alo = fminf(alo, fminf(fabsf(g[c]), fabsf(m[c])));
+        ahi = fmaxf(ahi, fmaxf(fabsf(g[c]), fabsf(m[c])));
+    }
+    const bool inrange = P.eps_inrange != 0u && vlo >= kSqrtLo && vhi <= kSqrtHi &&
+                         alo >= kDivNumLo && ahi <= kDivNumHi;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        float ug, um;
+        if (inrange) {
+            const float den = __fadd_rn(sqrt_rn_inrange(vh[c]), P.eps);
+            ug = div_rn_inrange(g[c], den);
+            um = div_rn_inrange(m[c], den);
+        } else {
+            ug = adam_quotient_anyrange(g[c], vh[c], P.eps);
+            um = adam_quotient_anyrange(m[c], vh[c], P.eps);
+        }
+        const float decayed = __fsub_rn(w[c], __fmul_rn(P.lrwd, w[c]));
+        what[c] = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug)), __fmul_rn(P.cm, um));
+    }
+}
+
+// NADAM: NAdamW and nothing else, decided at compile time (the owner kernel's form for the
+// paper's asynchronous-pipeline optimizer); GEN: either optimizer, decided by P.nesterov.
+template <bool GEN, int NC, bool NADAM = false>
 __device__ __forceinline__ void adamw_group(const StepParams &P, const float (&w)[NC],
                                             const float (&g)[NC], float (&m)[NC], float (&v)[NC],
                                             float (&what)[NC])
@@ -171,35 +206,12 @@ __device__ __forceinline__ void adamw_group(const StepParams &P, const float (&w
         mh[c] = __fmul_rn(m[c], P.ib1);
         vh[c] = __fmul_rn(v[c], P.ib2);
     }
-    if constexpr (GEN) {
+    if constexpr (NADAM) {
+        nadamw_finish<NC>(P, w, g, m, vh, what);
+        return;
+    } else if constexpr (GEN) {
         if (P.nesterov != 0u) {
-            // NAdamW (Appendix B.1): gradient part and (uncorrected) momentum part over
-            // the same denominator, weighted by the momentum schedule's cg and cm
-            float vlo = vh[0], vhi = vh[0], alo = fminf(fabsf(g[0]), fabsf(m[0])),
-                  ahi = fmaxf(fabsf(g[0]), fabsf(m[0]));
-#pragma unroll
-            for (int c = 1; c < NC; ++c) {
-                vlo = fminf(vlo, vh[c]);
-                vhi = fmaxf(vhi, vh[c]);
-                alo = fminf(alo, fminf(fabsf(g[c]), fabsf(m[c])));
-                ahi = fmaxf(ahi, fmaxf(fabsf(g[c]), fabsf(m[c])));
-            }
-            const bool inrange = P.eps_inrange != 0u && vlo >= kSqrtLo && vhi <= kSqrtHi &&
-                                 alo >= kDivNumLo && ahi <= kDivNumHi;
-#pragma unroll
-            for (int c = 0; c < NC; ++c) {
-                float ug, um;
-                if (inrange) {
-                    const float den = __fadd_rn(sqrt_rn_inrange(vh[c]), P.eps);
-                    ug = div_rn_inrange(g[c], den);
-                    um = div_rn_inrange(m[c], den);
-                } else {
-                    ug = adam_quotient_anyrange(g[c], vh[c], P.eps);
-                    um = adam_quotient_anyrange(m[c], vh[c], P.eps);
-                }
-                const float decayed = __fsub_rn(w[c], __fmul_rn(P.lrwd, w[c]));
-                what[c] = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug)), __fmul_rn(P.cm, um));
-            }
+            nadamw_finish<NC>(P, w, g, m, vh, what);
             return;
         }
     }

@@ -230,7 +230,8 @@ __device__ __forceinline__ float div_by_replicas(const StepParams &P, float a)
 // DIAG: the pass also accumulates the consensus error sum_i ||w_i - wbar||^2 of every stage (Section 3.3)
 // from the final weights it holds in registers anyway: no extra memory traffic, fp64 arithmetic per
 // coordinate, one atomicAdd per warp and stage.  A separate set of instantiations.
-template <int R, int RU, int V, int NST, int E, int MODE, bool GEN, bool DIAG = false>
+// NADAM: the common form with NAdamW in the place of AdamW (not together with GEN or DIAG).
+template <int R, int RU, int V, int NST, int E, int MODE, bool GEN, bool DIAG = false, bool NADAM = false>
 __global__ void __launch_bounds__(kOwnerThreads, R <= 4 ? kOwnerBlocksPerSM : 2)
 asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
 {
@@ -402,7 +403,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                         m[4 * h] = m4.x; m[4 * h + 1] = m4.y; m[4 * h + 2] = m4.z; m[4 * h + 3] = m4.w;
                         v[4 * h] = v4.x; v[4 * h + 1] = v4.y; v[4 * h + 2] = v4.z; v[4 * h + 3] = v4.w;
                     }
-                    adamw_group<GEN, NB>(P, wo[i], gg, m, v, wn[i]);
+                    adamw_group<GEN, NB, NADAM>(P, wo[i], gg, m, v, wn[i]);
 #pragma unroll
                     for (int h = 0; h < V; ++h) {
                         const uint64_t mu = mu0 + (uint64_t)h * 128;

@@ -1,13 +1,13 @@
-// Instantiations of the step kernels.  Compiled eleven times, -DAM_PART=0..10:
+// Instantiations of the step kernels.  Compiled twelve times, -DAM_PART=0..11:
 // 0 direct kernel R = 1..8; 1 direct kernel R = 9..16, common form; 2 the same,
 // general form; 3 / 4 pipelined kernel R = 1..8, common / general form; 5 / 6
 // pipelined kernel R = 9..16, common / general form; 7 / 8 / 9 owner kernel R = 1..8,
 // common / general / consensus-tracking form; 10 direct kernel with the dense ring kept as
-// exchanged (bfloat16 / E4M3 slots), R = 1..16, both forms.
+// exchanged (bfloat16 / E4M3 slots), R = 1..16, both forms; 11 owner kernel, common form with NAdamW.
 #include "kernel_table.cuh"
 
 #ifndef AM_PART
-#error "compile with -DAM_PART=0..10"
+#error "compile with -DAM_PART=0..11"
 #endif
 
 namespace amk {
@@ -108,12 +108,13 @@ KernelChoice pick_direct_many_general(uint32_t R, int mode)
 
 constexpr bool kGeneral = (AM_PART == 8);
 constexpr bool kTracking = (AM_PART == 9);   // the common form that also accumulates the consensus error
+constexpr bool kNadam = (AM_PART == 11);     // the common form with NAdamW as its optimizer
 
 template <int R, int E, int MODE>
 static KernelChoice owner_as(uint32_t S)
 {
     KernelChoice c;
-    c.fn = asyncmesh_step_kernel_owner<R, owner_ru(R), kOwnerV, owner_stages(MODE), E, MODE, kGeneral, kTracking>;
+    c.fn = asyncmesh_step_kernel_owner<R, owner_ru(R), kOwnerV, owner_stages(MODE), E, MODE, kGeneral, kTracking, kNadam>;
     c.threads = kOwnerThreads;
     c.smem = (size_t)pipe_table_bytes(S) +
              (size_t)(kOwnerThreads / 32) * OwnerCfg<R, owner_ru(R), kOwnerV, E>::warp_bytes(owner_stages(MODE));
@@ -132,8 +133,10 @@ static KernelChoice owner(int mode, int entries, uint32_t S)
 KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S)
 #elif AM_PART == 8
 KernelChoice pick_owner_general(uint32_t R, int mode, int entries, uint32_t S)
-#else
+#elif AM_PART == 9
 KernelChoice pick_owner_tracking(uint32_t R, int mode, int entries, uint32_t S)
+#else
+KernelChoice pick_owner_nadamw(uint32_t R, int mode, int entries, uint32_t S)
 #endif
 {
     switch (R) {

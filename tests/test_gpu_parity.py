@@ -205,7 +205,13 @@ def test_nadamw(tau, p):
              flags=binding.FLAG_DIRECT_KERNEL)
     run_case(6, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp)   # pipelined kernel
     run_case(4, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
-             flags=binding.FLAG_OWNER_KERNEL)
+             flags=binding.FLAG_OWNER_KERNEL)       # owner kernel, NAdamW form (the default for tau = 0)
+    run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
+             flags=binding.FLAG_PIPELINED_KERNEL)   # pipelined kernel, general form
+    run_case(2, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp, correction="eager",
+             flags=binding.FLAG_OWNER_KERNEL)       # owner kernel, general form
+    if tau == 0:
+        run_case(8, [6000, 77], p, tau, 0.9, steps=6, optimizer="nadamw", hp=hp)   # owner, two rows per unit
 
 
 @pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (3, 0.4)])
@@ -538,7 +544,14 @@ def test_kernel_name_tells_which_kernel_runs():
     assert mk(4, 1.0, 2) == "direct R=4 dense"
     assert mk(4, 1.0, 0) == "direct R=4 sync"
     assert mk(4, 0.05, 2, optimizer="nadamw") == "pipelined R=4 compact wide general"
-    assert mk(4, 0.05, 2, binding.FLAG_OWNER_KERNEL, optimizer="nadamw") == "owner R=4 compact entries=32 general"
+    assert mk(4, 0.05, 2, binding.FLAG_OWNER_KERNEL, optimizer="nadamw") == "owner R=4 compact entries=32 nadamw"
+    assert mk(4, 0.05, 0, optimizer="nadamw") == "owner R=4 sync nadamw"
+    assert mk(8, 0.05, 0, optimizer="nadamw") == "owner R=8 sync nadamw"
+    assert mk(8, 0.05, 2, optimizer="nadamw") == "pipelined R=8 compact wide general"
+    assert mk(4, 0.05, 2, binding.FLAG_PIPELINED_KERNEL, optimizer="nadamw") == "pipelined R=4 compact wide general"
+    assert mk(4, 0.05, 2, optimizer="nadamw", correction="eager") == "pipelined R=4 compact wide general"
+    assert mk(4, 0.05, 2, binding.FLAG_OWNER_KERNEL, correction="eager") == "owner R=4 compact entries=32 general"
+    assert mk(4, 0.05, 0, binding.FLAG_BF16_EXCHANGE, optimizer="nadamw") == "owner R=4 sync nadamw"
 
 
 def test_init_from_device_tensor_and_bad_state():
