@@ -580,24 +580,22 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     // unless a flag asks for another kernel.  1B layout, tau = 4, ms per step, pipelined
     // against owner: p = 0.01 21.6 / 20.7, 0.05 23.4 / 22.7, 0.1 26.2 / 23.9, 0.25 30.9 / 25.6,
     // 0.5 37.4 / 29.0; tau = 0: 20.8 to 24.4 / 20.5 to 20.7 at every p.
-    // E4M3 exchange, the eager estimate and NAdamW: the kernels' general form.  The owner
-    // kernel carries that form's optimizer code four times over (once per unit of a
-    // group) and loses more to it than the pipelined kernel does (1B layout, NAdamW: 30.1
-    // against 24.1 ms per step), so the general form stays with the pipelined kernel.
+    // E4M3 exchange, the eager estimate and NAdamW: the kernels' general form.  With the ring the
+    // owner kernel loses more to that form than the pipelined kernel does (1B layout, E4M3 exchange:
+    // 26.9 against 23.4 ms per step at p = 0.05, 33.6 against 30.4 at p = 0.25), so there the general
+    // form stays with the pipelined kernel; for tau = 0 the owner kernel keeps its lead (19.3 against 20.7).
     // (a ring kept as exchanged converts by its slot format, which is a template parameter: common form)
     const bool general = (h->wire == 2u && h->mode <= kDense) || h->correction == ASYNCMESH_CORRECTION_EAGER ||
                          h->optimizer == ASYNCMESH_OPT_NADAMW;
     // NAdamW alone (the optimizer of the paper's asynchronous-pipeline runs) has an owner form of its
-    // own, with the optimizer fixed at compile time.  1B layout, ms per step, that form against the
-    // pipelined kernel's general form: tau = 0 19.56 / 21.34, so it is the default there; with the ring
-    // 26.2 / 24.3 at p = 0.05 and 32.1 / 30.0 at p = 0.25 (the second division costs the owner kernel,
-    // which has no registers to spare at three blocks per SM, more than it costs the pipelined one):
-    // there only on ASYNCMESH_FLAG_OWNER_KERNEL, where it replaces the general form's 30.1.
+    // own, with the optimizer fixed at compile time, and goes where AdamW goes.  1B layout, ms per step,
+    // that form against the pipelined kernel's general form: tau = 0 19.1 / 20.9; tau = 4, p = 0.05
+    // 22.6 / 23.3, p = 0.25 27.1 / 29.7 (AdamW in the owner kernel: 19.1, 22.5, 25.6).
     const bool nadam_only = h->optimizer == ASYNCMESH_OPT_NADAMW && h->wire != 2u &&
                             h->correction != ASYNCMESH_CORRECTION_EAGER;
     const bool owner_asked = (cfg->flags & ASYNCMESH_FLAG_OWNER_KERNEL) != 0;
     const bool owner_default =
-        (!general || (nadam_only && h->mode == kSync)) && !(cfg->flags & (ASYNCMESH_FLAG_DIRECT_KERNEL | ASYNCMESH_FLAG_PIPELINED_KERNEL)) &&
+        (!general || nadam_only || h->mode == kSync) && !(cfg->flags & (ASYNCMESH_FLAG_DIRECT_KERNEL | ASYNCMESH_FLAG_PIPELINED_KERNEL)) &&
         (h->mode == kCompact || (h->mode == kSync && cfg->p <= 0.8));
     // (five to eight replicas: for tau = 0 only; 350M layout, p = 0.05: 14.15 against 15.09 ms, while with
     // the ring the pipelined kernel is as fast at p = 0.05 and faster at p = 0.01 and 0.25)

@@ -175,19 +175,25 @@ __device__ __forceinline__ void nadamw_finish(const StepParams &P, const float (
     }
     const bool inrange = P.eps_inrange != 0u && vlo >= kSqrtLo && vhi <= kSqrtHi &&
                          alo >= kDivNumLo && ahi <= kDivNumHi;
+    float ug[NC], um[NC];
+    if (inrange) {   // one branch for the group: the chains of its coordinates interleave
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const float den = __fadd_rn(sqrt_rn_inrange(vh[c]), P.eps);
+            ug[c] = div_rn_inrange(g[c], den);
+            um[c] = div_rn_inrange(m[c], den);
+        }
+    } else {
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            ug[c] = adam_quotient_anyrange(g[c], vh[c], P.eps);
+            um[c] = adam_quotient_anyrange(m[c], vh[c], P.eps);
+        }
+    }
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
-        float ug, um;
-        if (inrange) {
-            const float den = __fadd_rn(sqrt_rn_inrange(vh[c]), P.eps);
-            ug = div_rn_inrange(g[c], den);
-            um = div_rn_inrange(m[c], den);
-        } else {
-            ug = adam_quotient_anyrange(g[c], vh[c], P.eps);
-            um = adam_quotient_anyrange(m[c], vh[c], P.eps);
-        }
         const float decayed = __fsub_rn(w[c], __fmul_rn(P.lrwd, w[c]));
-        what[c] = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug)), __fmul_rn(P.cm, um));
+        what[c] = __fsub_rn(__fsub_rn(decayed, __fmul_rn(P.cg, ug[c])), __fmul_rn(P.cm, um[c]));
     }
 }
 

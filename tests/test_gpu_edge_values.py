@@ -144,7 +144,7 @@ def test_edge_values_with_the_ring_kept_as_exchanged(exchange, R):
 
 
 def test_edge_values_nadamw():
-    run(4, 2 * 1024 + 7, 0.3, 2, 0, optimizer="nadamw")                          # pipelined kernel, general form
-    run(4, 2 * 1024 + 7, 0.3, 2, flags_of("owner"), optimizer="nadamw")          # owner kernel, NAdamW form
+    run(4, 2 * 1024 + 7, 0.3, 2, 0, optimizer="nadamw")                          # owner kernel, NAdamW form
+    run(4, 2 * 1024 + 7, 0.3, 2, flags_of("pipelined"), optimizer="nadamw")      # pipelined kernel, general form
     run(4, 2 * 1024 + 7, 0.3, 0, 0, optimizer="nadamw", steps=4)
     run(8, 2 * 1024 + 7, 0.3, 2, 0, optimizer="nadamw")

@@ -205,7 +205,7 @@ def test_nadamw(tau, p):
              flags=binding.FLAG_DIRECT_KERNEL)
     run_case(6, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp)   # pipelined kernel
     run_case(4, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
-             flags=binding.FLAG_OWNER_KERNEL)       # owner kernel, NAdamW form (the default for tau = 0)
+             flags=binding.FLAG_OWNER_KERNEL)       # owner kernel, NAdamW form (the default where AdamW has the owner kernel)
     run_case(4, [6000, 1024 + 9], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp,
              flags=binding.FLAG_PIPELINED_KERNEL)   # pipelined kernel, general form
     run_case(2, [6000], p, tau, 0.9, steps=3 * tau + 6, optimizer="nadamw", hp=hp, correction="eager",
@@ -543,10 +543,13 @@ def test_kernel_name_tells_which_kernel_runs():
     assert mk(4, 0.05, 2, binding.FLAG_DIRECT_KERNEL) == "direct R=4 compact"
     assert mk(4, 1.0, 2) == "direct R=4 dense"
     assert mk(4, 1.0, 0) == "direct R=4 sync"
-    assert mk(4, 0.05, 2, optimizer="nadamw") == "pipelined R=4 compact wide general"
-    assert mk(4, 0.05, 2, binding.FLAG_OWNER_KERNEL, optimizer="nadamw") == "owner R=4 compact entries=32 nadamw"
+    assert mk(4, 0.05, 2, optimizer="nadamw") == "owner R=4 compact entries=32 nadamw"
+    assert mk(4, 0.3, 2, optimizer="nadamw") == "owner R=4 compact entries=128 nadamw"
     assert mk(4, 0.05, 0, optimizer="nadamw") == "owner R=4 sync nadamw"
     assert mk(8, 0.05, 0, optimizer="nadamw") == "owner R=8 sync nadamw"
+    assert mk(4, 0.3, 0, binding.FLAG_FP8_EXCHANGE) == "owner R=4 sync general"
+    assert mk(6, 0.3, 0, correction="eager") == "owner R=6 sync general"
+    assert mk(4, 0.05, 2, binding.FLAG_FP8_EXCHANGE) == "pipelined R=4 compact wide general"
     assert mk(8, 0.05, 2, optimizer="nadamw") == "pipelined R=8 compact wide general"
     assert mk(4, 0.05, 2, binding.FLAG_PIPELINED_KERNEL, optimizer="nadamw") == "pipelined R=4 compact wide general"
     assert mk(4, 0.05, 2, optimizer="nadamw", correction="eager") == "pipelined R=4 compact wide general"
