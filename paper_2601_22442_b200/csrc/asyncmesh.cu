@@ -599,10 +599,16 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
         (h->mode == kCompact || (h->mode == kSync && cfg->p <= 0.8));
     // (five to eight replicas: for tau = 0 only; 350M layout, p = 0.05: 14.15 against 15.09 ms, while with
     // the ring the pipelined kernel is as fast at p = 0.05 and faster at p = 0.01 and 0.25)
-    if ((R <= 4 || (R <= 8 && h->mode == kSync)) && !is_dense(h->mode) && (owner_asked || owner_default)) {
-        const double mean = 128.0 * kOwnerV * cfg->p, sd = std::sqrt(mean * (1.0 - cfg->p));
-        h->pipelined = h->mode == kSync ? 6 : (mean + 4.0 * sd <= (double)kOwnerEntriesFew ? 4 : 5);
-    }
+    // Six and eight replicas with the ring: two passes of three and four replicas over each group.  350M
+    // layout (R = 8, tau = 4), ms per step, pipelined against that: p = 0.01 14.51 / 14.47, 0.05 15.73 / 15.66,
+    // 0.25 20.15 / 18.80, 0.5 21.93 / 21.80; 125M layout (tau = 2): 4.66 / 4.68, 5.03 / 5.06, 6.43 / 6.02.
+    // The default where it wins: the subsets that need the many-entries form.
+    const bool two_pass = (R == 6 || R == 8) && h->mode == kCompact;
+    const double group_mean = 128.0 * kOwnerV * cfg->p;
+    const bool few_entries = group_mean + 4.0 * std::sqrt(group_mean * (1.0 - cfg->p)) <= (double)kOwnerEntriesFew;
+    if ((R <= 4 || (R <= 8 && h->mode == kSync) || two_pass) && !is_dense(h->mode) &&
+        (owner_asked || (owner_default && (!two_pass || !few_entries))))
+        h->pipelined = h->mode == kSync ? 6 : (few_entries ? 4 : 5);
 
 
     auto bail = [&](int code, const char *what) {
@@ -683,7 +689,8 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     h->kernel = h->nadam_form
         ? pick_owner_nadamw(R, h->mode, h->pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany, S)
         : pick_kernel(R, h->mode, h->pipelined, general, S);
-    if ((cfg->flags & ASYNCMESH_FLAG_TRACK_CONSENSUS) && h->pipelined >= 4 && !general) {
+    if ((cfg->flags & ASYNCMESH_FLAG_TRACK_CONSENSUS) && h->pipelined >= 4 && !general &&
+        (R <= 4 || h->mode == kSync)) {
         h->tracking = true;
         h->kernel = pick_owner_tracking(R, h->mode, h->pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany, S);
     }

@@ -28,7 +28,7 @@ KernelChoice pick_pipelined_few_common(uint32_t R, int shape, uint32_t S);     /
 KernelChoice pick_pipelined_few_general(uint32_t R, int shape, uint32_t S);
 KernelChoice pick_pipelined_many_common(uint32_t R, int shape, uint32_t S);    // R = 9..16
 KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S);
-// Owner kernel (R = 1..4; R = 5..8 for kSync only).  mode: kCompact or kSync; entries: ring / d entries per group
+// Owner kernel (R = 1..4; R = 5..8 for kSync; R = 6 and 8 for kCompact as two passes over each group).  mode: kCompact or kSync; entries: ring / d entries per group
 // of 256 coordinates fetched ahead (kOwnerEntriesFew or kOwnerEntriesMany).
 // Shape, measured on the 1B layout (R = 4, p = 0.05, ms per step): one replica row per
 // unit and 8 coordinates per lane (1 KB contiguous per array row and request) 22.7;

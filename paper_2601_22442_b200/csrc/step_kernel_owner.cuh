@@ -1,4 +1,5 @@
-// Third form of the fused step, for few replicas (up to four; up to eight for tau = 0):
+// Third form of the fused step, for few replicas (up to four; up to eight for tau = 0; six and
+// eight with the ring as two passes of three and four, see NH below):
 // the lane that owns a coordinate does all of its work, sparse part included, and
 // nothing is handed from lane to lane.  Same results as the other two kernels, bit
 // for bit.
@@ -58,17 +59,21 @@ __device__ __forceinline__ void cp_async_replicas(uint32_t smem_addr, const floa
 // RU: replica rows per pipeline unit (divides R); V: float4 per lane, array row and unit;
 // E: coordinates per group whose ring and d entries are fetched ahead (further ones,
 // possible only when p is large for the E chosen, are read in place).
-template <int R, int RU, int V, int E>
+// NH: passes over a group.  A lane holds R replicas at a time; with NH > 1 the stage has R NH replicas
+// and a group is walked NH times, R replica rows per pass (the ring entry carries all of them for the
+// mean, d and the snapshot move in the pass's own part).
+template <int R, int RU, int V, int E, int NH = 1>
 struct OwnerCfg {
     static_assert(R % RU == 0, "a unit holds whole replica rows");
-    static constexpr int kUnitsPerGroup = R / RU;
+    static constexpr int kTotal = R * NH;                            // replicas of the stage
+    static constexpr int kUnitsPerGroup = R / RU;                    // per pass
     static constexpr int kBits = 4 * V;                              // mask bits per lane and group
     static constexpr int kGroupCoords = 128 * V;
     static constexpr int kGroups = kWarpChunk / kGroupCoords;
     static constexpr int kUnitBytes = 4 * RU * V * 512;              // w, g, m, v
-    static constexpr bool kPair = (R == 4);                          // d moves as 32-byte pairs
-    static constexpr int kOldFloats = (R + 3) / 4 * 4;               // ring entry, padded to 16 bytes
-    static constexpr int kDFloats = kPair ? 8 : kOldFloats;
+    static constexpr bool kPair = (R == 4 && NH == 1);               // d moves as 32-byte pairs
+    static constexpr int kOldFloats = (kTotal + 3) / 4 * 4;          // ring entry, padded to 16 bytes
+    static constexpr int kDFloats = kPair ? 8 : (R + 3) / 4 * 4;     // d of the pass's replicas
     static constexpr int kEntryFloats = kOldFloats + kDFloats;
     static constexpr int kSparseBytes = E * kEntryFloats * 4;
     __host__ __device__ static constexpr int sparse_areas(int stages)
@@ -89,7 +94,8 @@ struct OwnerCfg {
 struct OwnerCursor {
     uint64_t mu;                 // first coordinate of this lane in the current group
     uint32_t gc, s;
-    int g, gmax;
+    int g, gmax;                 // passes over groups done in this chunk / in all (groups x NH)
+    uint32_t h;                  // pass over the current group
     bool valid;
     uint32_t cmask, cbase, crun; // consumed coordinates of the chunk: lane's mask, slot base, count before group g
     uint32_t nx_cmask, nx_cbase; // the same two for the warp's next chunk, asked for one chunk ahead
@@ -117,7 +123,7 @@ __device__ __forceinline__ int owner_groups(uint64_t N, uint32_t chunk)
     return rem >= (uint64_t)kWarpChunk ? kWarpChunk / GC : (int)((rem + GC - 1) / GC);
 }
 
-template <int GC>
+template <int GC, int NH = 1>
 __device__ __forceinline__ void owner_enter_chunk(OwnerCursor &c, const StepParams &P,
                                                   const StageDesc *sd, int lane, uint32_t n_warps,
                                                   bool consume)
@@ -127,8 +133,9 @@ __device__ __forceinline__ void owner_enter_chunk(OwnerCursor &c, const StepPara
     while (c.s + 1 < P.S && c.gc >= sd[c.s + 1].chunk_begin) ++c.s;
     const StageDesc &st = sd[c.s];
     const uint32_t chunk = c.gc - st.chunk_begin;
-    c.gmax = owner_groups<GC>(st.N, chunk);
+    c.gmax = owner_groups<GC>(st.N, chunk) * NH;
     c.g = 0;
+    c.h = 0;
     c.mu = (uint64_t)chunk * kWarpChunk + (uint64_t)lane * 4;
     if (consume) {
         c.cbase = c.nx_cbase;
@@ -156,14 +163,15 @@ __device__ __forceinline__ uint32_t owner_ranks(uint32_t m, uint32_t lt, uint32_
 // CU: which unit of its group the cursor is at.  The cursor runs a fixed NST - 1 units
 // ahead of the arithmetic, whose unit loop is unrolled, so CU is known at compile time
 // and the code that only a group's first or last unit needs exists once.
-template <int R, int RU, int V, int E, int NST, int CU>
+template <int R, int RU, int V, int E, int NST, int CU, int NH = 1>
 __device__ __forceinline__ void owner_issue_unit(OwnerCursor &c, const StepParams &P,
                                                  const StageDesc *sd, uint32_t stage_addr,
                                                  uint32_t sparse_base, int lane, uint32_t lt,
                                                  uint32_t n_warps, bool consume)
 {
-    using Cfg = OwnerCfg<R, RU, V, E>;
+    using Cfg = OwnerCfg<R, RU, V, E, NH>;
     constexpr int NB = Cfg::kBits;
+    constexpr int RT = Cfg::kTotal;
     if (c.valid) {
         const StageDesc &st = sd[c.s];
         const uint32_t a = stage_addr + lane * 16;
@@ -174,7 +182,7 @@ __device__ __forceinline__ void owner_issue_unit(OwnerCursor &c, const StepParam
             if (mu < st.N) {
 #pragma unroll
                 for (int ii = 0; ii < RU; ++ii) {
-                    const uint64_t off = (uint64_t)(CU * RU + ii) * st.stride + mu;
+                    const uint64_t off = (uint64_t)(c.h * R + CU * RU + ii) * st.stride + mu;
                     cp_async16(a + ((0 * RU + ii) * V + h) * 512, st.W + off);
                     cp_async16(a + ((1 * RU + ii) * V + h) * 512, G + off);
                     cp_async16(a + ((2 * RU + ii) * V + h) * 512, st.M + off);
@@ -184,7 +192,7 @@ __device__ __forceinline__ void owner_issue_unit(OwnerCursor &c, const StepParam
         }
         if (CU == 0 && consume) {   // the group's ring and d entries ride with its first unit
             constexpr uint32_t kGroupMask = NB == 32 ? 0xFFFFFFFFu : ((1u << (NB % 32)) - 1u);
-            const uint32_t cm = (c.cmask >> (NB * c.g)) & kGroupMask;
+            const uint32_t cm = (c.cmask >> (NB * (c.g / NH))) & kGroupMask;
             uint32_t e[NB];
             const uint32_t total = owner_ranks<NB>(cm, lt, e);
             if (cm) {
@@ -195,22 +203,25 @@ __device__ __forceinline__ void owner_issue_unit(OwnerCursor &c, const StepParam
                     if (((cm >> j) & 1u) && e[j] < (uint32_t)E) {
                         const uint32_t dst = sp + e[j] * (Cfg::kEntryFloats * 4);
                         const uint64_t coord = c.mu + (uint64_t)(j >> 2) * 128 + (j & 3);
-                        cp_async_replicas<R>(dst, ring_cons + (uint64_t)(c.cbase + c.crun + e[j]) * R);
+                        cp_async_replicas<RT>(dst, ring_cons + (uint64_t)(c.cbase + c.crun + e[j]) * RT);
                         if constexpr (Cfg::kPair)   // the whole sector: this coordinate's d and its pair's
                             cp_async_replicas<8>(dst + Cfg::kOldFloats * 4, st.D + (coord & ~(uint64_t)1) * R);
                         else
-                            cp_async_replicas<R>(dst + Cfg::kOldFloats * 4, st.D + coord * R);
+                            cp_async_replicas<R>(dst + Cfg::kOldFloats * 4, st.D + coord * RT + c.h * R);
                     }
                 }
             }
-            c.crun += total;
+            if (NH == 1 || c.h == NH - 1) c.crun += total;
         }
         if constexpr (CU == Cfg::kUnitsPerGroup - 1) {
-            c.mu += Cfg::kGroupCoords;
+            if (NH == 1 || ++c.h == NH) {   // the group's last pass
+                c.h = 0;
+                c.mu += Cfg::kGroupCoords;
+            }
             c.sp = (c.sp + 1 == (uint32_t)Cfg::sparse_areas(NST)) ? 0u : c.sp + 1;
             if (++c.g == c.gmax) {
                 c.gc += n_warps;
-                owner_enter_chunk<Cfg::kGroupCoords>(c, P, sd, lane, n_warps, consume);
+                owner_enter_chunk<Cfg::kGroupCoords, NH>(c, P, sd, lane, n_warps, consume);
             }
         }
     }
@@ -231,12 +242,16 @@ __device__ __forceinline__ float div_by_replicas(const StepParams &P, float a)
 // from the final weights it holds in registers anyway: no extra memory traffic, fp64 arithmetic per
 // coordinate, one atomicAdd per warp and stage.  A separate set of instantiations.
 // NADAM: the common form with NAdamW in the place of AdamW (not together with GEN or DIAG).
-template <int R, int RU, int V, int NST, int E, int MODE, bool GEN, bool DIAG = false, bool NADAM = false>
+// NH: the stage has R NH replicas, a group is walked NH times (see OwnerCfg; compact ring only).
+template <int R, int RU, int V, int NST, int E, int MODE, bool GEN, bool DIAG = false, bool NADAM = false,
+          int NH = 1>
 __global__ void __launch_bounds__(kOwnerThreads, R <= 4 ? kOwnerBlocksPerSM : 2)
 asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
 {
     static_assert(MODE == kCompact || MODE == kSync, "compact ring or synchronous");
-    using Cfg = OwnerCfg<R, RU, V, E>;
+    static_assert(NH == 1 || (MODE == kCompact && !DIAG), "several passes: the mean comes from the ring entry");
+    using Cfg = OwnerCfg<R, RU, V, E, NH>;
+    constexpr int RT = Cfg::kTotal;
     constexpr int NB = Cfg::kBits;
     constexpr int UPG = Cfg::kUnitsPerGroup;
     constexpr int kUnitBytes = Cfg::kUnitBytes;
@@ -273,14 +288,14 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
     pf.cmask = pf.cbase = pf.crun = 0;
     pf.sp = 0;
     if (consume) owner_peek(P, sd, pf.gc, 0u, lane, pf.nx_cbase, pf.nx_cmask);
-    owner_enter_chunk<Cfg::kGroupCoords>(pf, P, sd, lane, n_warps, consume);
+    owner_enter_chunk<Cfg::kGroupCoords, NH>(pf, P, sd, lane, n_warps, consume);
     static_assert(NST == 2 || NST == 3 || NST == 4, "the prologue below issues one to three units");
-    owner_issue_unit<R, RU, V, E, NST, 0>(pf, P, sd, stage_base, sparse_base, lane, lt, n_warps, consume);
+    owner_issue_unit<R, RU, V, E, NST, 0, NH>(pf, P, sd, stage_base, sparse_base, lane, lt, n_warps, consume);
     if constexpr (NST >= 3)
-        owner_issue_unit<R, RU, V, E, NST, 1 % UPG>(pf, P, sd, stage_base + kUnitBytes, sparse_base, lane, lt,
+        owner_issue_unit<R, RU, V, E, NST, 1 % UPG, NH>(pf, P, sd, stage_base + kUnitBytes, sparse_base, lane, lt,
                                                     n_warps, consume);
     if constexpr (NST >= 4)
-        owner_issue_unit<R, RU, V, E, NST, 2 % UPG>(pf, P, sd, stage_base + 2 * kUnitBytes, sparse_base, lane,
+        owner_issue_unit<R, RU, V, E, NST, 2 % UPG, NH>(pf, P, sd, stage_base + 2 * kUnitBytes, sparse_base, lane,
                                                     lt, n_warps, consume);
     uint32_t rd = 0, wr = NST - 1;   // stage being consumed / being filled
     uint32_t sp_rd = 0;              // sparse area of the group being computed
@@ -289,7 +304,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
     auto advance = [&](auto cu_tag) -> const unsigned char * {
         constexpr int CU = decltype(cu_tag)::value;
         cp_async_wait<NST - 2>();
-        owner_issue_unit<R, RU, V, E, NST, CU>(pf, P, sd, stage_base + wr * kUnitBytes, sparse_base, lane, lt,
+        owner_issue_unit<R, RU, V, E, NST, CU, NH>(pf, P, sd, stage_base + wr * kUnitBytes, sparse_base, lane, lt,
                                                n_warps, consume);
         const unsigned char *slot = my + rd * kUnitBytes + lane * 16;
         rd = (rd + 1 == NST) ? 0 : rd + 1;
@@ -376,7 +391,10 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
         uint32_t crun = 0, prun = 0;
 
 #pragma unroll 1
-        for (int g = 0; g < gmax; ++g) {
+        for (int vg = 0; vg < gmax * NH; ++vg) {
+            const int g = vg / NH;                         // the group, and which R of its replica rows
+            const uint32_t row0 = (uint32_t)(vg % NH) * R;
+            const bool last_pass = NH == 1 || (vg % NH) == NH - 1;
             const uint64_t mu0 = c0 + (uint64_t)g * Cfg::kGroupCoords;   // h = 0; h adds 128
             const uint32_t pm = (pmask >> (NB * g)) & kGroupMask;
             const uint32_t cm = (cmask >> (NB * g)) & kGroupMask;
@@ -408,7 +426,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                     for (int h = 0; h < V; ++h) {
                         const uint64_t mu = mu0 + (uint64_t)h * 128;
                         if (mu < N) {
-                            const uint64_t off = (uint64_t)i * stride + mu;
+                            const uint64_t off = (uint64_t)(row0 + i) * stride + mu;
                             __stcs(reinterpret_cast<float4 *>(st.M + off),
                                    make_float4(m[4 * h], m[4 * h + 1], m[4 * h + 2], m[4 * h + 3]));
                             __stcs(reinterpret_cast<float4 *>(st.V + off),
@@ -437,7 +455,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                         // with one lane taking part as with all of them, and most lanes have at
                         // most one entry per group: a lane holds its first entry back, so that one
                         // store instruction at the end serves the first entries of all lanes.
-                        float *ring_at = ring_prod + (uint64_t)(pbase + prun) * R;
+                        float *ring_at = ring_prod + (uint64_t)(pbase + prun) * RT + row0;
                         float held[R];
                         uint32_t held_e = kInvalidBase;
 #pragma unroll
@@ -451,13 +469,13 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
 #pragma unroll
                                     for (int i = 0; i < R; ++i) held[i] = x[i];
                                 } else {
-                                    store_replicas<R>(ring_at + (uint64_t)e[j] * R, x);
+                                    store_replicas<R>(ring_at + (uint64_t)e[j] * RT, x);
                                 }
                             }
                         }
-                        store_replicas<R>(ring_at + (uint64_t)held_e * R, held);
+                        store_replicas<R>(ring_at + (uint64_t)held_e * RT, held);
                     }
-                    prun += total;
+                    if (last_pass) prun += total;
                 }
                 // ---- Eq. "asparta" / Eq. "ema" + corrected averaging on S^{t-tau} --------
                 if (consume) {
@@ -466,11 +484,12 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                     if (cm) {
                         const float *sp = reinterpret_cast<const float *>(my_sparse + sp_rd * Cfg::kSparseBytes);
                         // one consumed coordinate: stale average from the ring entry, new d, final w
-                        auto consume_one = [&](int j, const float (&old)[R], float (&dd)[R]) {
-                            float a = on_wire<GEN>(P, old[0]);
+                        // (all: the ring entry, every replica of the stage; old: the values of this pass's replicas)
+                        auto consume_one = [&](int j, const float (&all)[RT], const float (&old)[R], float (&dd)[R]) {
+                            float a = on_wire<GEN>(P, all[0]);
 #pragma unroll
-                            for (int i = 1; i < R; ++i) a = __fadd_rn(a, on_wire<GEN>(P, old[i]));
-                            const float abar = div_by_replicas<R>(P, a);
+                            for (int i = 1; i < RT; ++i) a = __fadd_rn(a, on_wire<GEN>(P, all[i]));
+                            const float abar = div_by_replicas<RT>(P, a);
 #pragma unroll
                             for (int i = 0; i < R; ++i) {
                                 const float diff = __fsub_rn(wn[i][j], old[i]);
@@ -500,7 +519,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                                             else load_replicas<R>(ring_cons + (uint64_t)(cbase + crun + e[j]) * R, old);
 #pragma unroll
                                             for (int i = 0; i < R; ++i) dd[i] = dpair[R * c + i];
-                                            consume_one(j, old, dd);
+                                            if constexpr (NH == 1) consume_one(j, old, old, dd);
 #pragma unroll
                                             for (int i = 0; i < R; ++i) dpair[R * c + i] = dd[i];
                                         }
@@ -519,22 +538,27 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
 #pragma unroll
                             for (int j = 0; j < NB; ++j) {
                                 if ((cm >> j) & 1u) {
-                                    float old[R], dd[R];
-                                    float *dp = st.D + (mu0 + (uint64_t)(j >> 2) * 128 + (j & 3)) * R;
+                                    float all[RT], old[NH == 1 ? 1 : R], dd[R];
+                                    float *dp = st.D + (mu0 + (uint64_t)(j >> 2) * 128 + (j & 3)) * RT + row0;
                                     if (e[j] < (uint32_t)E) {
-                                        load_replicas<R>(sp + e[j] * Cfg::kEntryFloats, old);
-                                        load_replicas<R>(sp + e[j] * Cfg::kEntryFloats + Cfg::kOldFloats, dd);
+                                        const float *entry = sp + e[j] * Cfg::kEntryFloats;
+                                        load_replicas<RT>(entry, all);
+                                        if constexpr (NH > 1) load_replicas<R>(entry + row0, old);
+                                        load_replicas<R>(entry + Cfg::kOldFloats, dd);
                                     } else {   // beyond what was fetched ahead
-                                        load_replicas<R>(ring_cons + (uint64_t)(cbase + crun + e[j]) * R, old);
+                                        const float *entry = ring_cons + (uint64_t)(cbase + crun + e[j]) * RT;
+                                        load_replicas<RT>(entry, all);
+                                        if constexpr (NH > 1) load_replicas<R>(entry + row0, old);
                                         load_replicas<R>(dp, dd);
                                     }
-                                    consume_one(j, old, dd);
+                                    if constexpr (NH == 1) consume_one(j, all, all, dd);
+                                    else consume_one(j, all, old, dd);
                                     store_replicas<R>(dp, dd);
                                 }
                             }
                         }
                     }
-                    crun += total;
+                    if (last_pass) crun += total;
                     sp_rd = (sp_rd + 1 == (uint32_t)Cfg::sparse_areas(NST)) ? 0u : sp_rd + 1;
                 }
             } else {
@@ -578,7 +602,7 @@ asyncmesh_step_kernel_owner(const __grid_constant__ StepParams P)
                 if (mu < N) {
 #pragma unroll
                     for (int i = 0; i < R; ++i) {
-                        const uint64_t off = (uint64_t)i * stride + mu;
+                        const uint64_t off = (uint64_t)(row0 + i) * stride + mu;
                         __stcs(reinterpret_cast<float4 *>(st.W + off),
                                make_float4(wn[i][4 * h], wn[i][4 * h + 1], wn[i][4 * h + 2], wn[i][4 * h + 3]));
                         if (has_look) {

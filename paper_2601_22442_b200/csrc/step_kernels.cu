@@ -121,6 +121,28 @@ static KernelChoice owner_as(uint32_t S)
     return c;
 }
 
+// Twice as many replicas as a lane holds: two passes over each group (compact ring; not the tracking form).
+template <int RH, int E>
+static KernelChoice owner_two_passes_as(uint32_t S)
+{
+    KernelChoice c;
+    if constexpr (!kTracking) {
+        c.fn = asyncmesh_step_kernel_owner<RH, owner_ru(RH), kOwnerV, owner_stages(kCompact), E, kCompact, kGeneral,
+                                           false, kNadam, 2>;
+        c.threads = kOwnerThreads;
+        c.smem = (size_t)pipe_table_bytes(S) +
+                 (size_t)(kOwnerThreads / 32) *
+                     OwnerCfg<RH, owner_ru(RH), kOwnerV, E, 2>::warp_bytes(owner_stages(kCompact));
+    }
+    return c;
+}
+template <int RH>
+static KernelChoice owner_two_passes(int entries, uint32_t S)
+{
+    return entries == kOwnerEntriesFew ? owner_two_passes_as<RH, kOwnerEntriesFew>(S)
+                                       : owner_two_passes_as<RH, kOwnerEntriesMany>(S);
+}
+
 template <int R>
 static KernelChoice owner(int mode, int entries, uint32_t S)
 {
@@ -144,11 +166,12 @@ KernelChoice pick_owner_nadamw(uint32_t R, int mode, int entries, uint32_t S)
     case 2: return owner<2>(mode, entries, S);
     case 3: return owner<3>(mode, entries, S);
     case 4: return owner<4>(mode, entries, S);
-    // five to eight replicas: the synchronous mode only (with the ring the pipelined kernel is as fast or faster)
+    // five to eight replicas: all of them in registers for the synchronous mode only; with the ring, six
+    // and eight replicas as two passes of three and four
     case 5: return mode == kSync ? owner_as<5, 1, kSync>(S) : KernelChoice();
-    case 6: return mode == kSync ? owner_as<6, 1, kSync>(S) : KernelChoice();
+    case 6: return mode == kSync ? owner_as<6, 1, kSync>(S) : owner_two_passes<3>(entries, S);
     case 7: return mode == kSync ? owner_as<7, 1, kSync>(S) : KernelChoice();
-    case 8: return mode == kSync ? owner_as<8, 1, kSync>(S) : KernelChoice();
+    case 8: return mode == kSync ? owner_as<8, 1, kSync>(S) : owner_two_passes<4>(entries, S);
     default: return KernelChoice();
     }
 }

@@ -125,7 +125,8 @@ RAGGED = [1, 3, 4, 5, 127, 128, 129, 1023, 1024, 1025, 4099]
 @pytest.mark.parametrize("R,p,tau,flags", [
     (2, 0.5, 1, 0), (4, 0.05, 2, 0), (4, 0.3, 2, 0), (3, 0.2, 0, 0), (4, 1.0, 0, 0), (4, 1.0, 2, 0),
     (8, 0.05, 2, 0), (8, 0.3, 1, 0), (5, 0.3, 0, 0), (4, 0.05, 2, 2), (4, 0.4, 2, 4), (4, 0.4, 0, 4),
-    (4, 0.3, 2, 32), (1, 0.3, 2, 0), (2, 0.9, 2, 256), (4, 0.9, 3, 256), (3, 0.6, 1, 256)])
+    (4, 0.3, 2, 32), (1, 0.3, 2, 0), (2, 0.9, 2, 256), (4, 0.9, 3, 256), (3, 0.6, 1, 256),
+    (8, 0.05, 2, 256), (6, 0.4, 2, 256), (8, 1.0, 1, 256), (8, 0.3, 1, 4)])
 def test_ragged_stage_sizes_keep_inside_their_blocks(R, p, tau, flags):
     run(R, RAGGED, p, tau, flags)
 

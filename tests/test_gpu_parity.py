@@ -167,14 +167,36 @@ def test_replica_counts(R):
 
 @pytest.mark.parametrize("flag", ["direct", "pipelined", "owner"])
 @pytest.mark.parametrize("R,p", [(4, 0.05), (8, 0.05), (3, 0.1), (4, 0.5), (8, 0.35), (2, 1.0), (5, 0.9),
-                                 (1, 0.3), (4, 1.0)])
+                                 (1, 0.3), (4, 1.0), (6, 0.05), (6, 0.6), (8, 1.0)])
 def test_all_compact_ring_kernels(flag, R, p):
     # the register-load kernel, the shared-memory pipelined kernel and the owner kernel are
     # three routes to the same numbers; large p forces the pipelined kernel through its
     # in-place path (more selected coordinates per sub-iteration than its stash holds) and
-    # the owner kernel past the ring / d entries it fetches ahead
+    # the owner kernel past the ring / d entries it fetches ahead; with six and eight replicas
+    # the owner kernel walks every group twice, half of the replicas per pass (with five, and
+    # with seven, the flag changes nothing)
     f = kernel_flag(flag)
     run_case(R, [9000, 1024 * 3 + 5, 77], p, 2, 0.9, steps=7, flags=f)
+
+
+def test_two_pass_owner_kernel_features():
+    from paper_2601_22442_b200 import binding
+    f = binding.FLAG_OWNER_KERNEL
+    sizes = [1, 3, 4, 5, 127, 128, 129, 1023, 1024, 1025, 4099]
+    run_case(8, sizes, 0.4, 3, 0.7, steps=8, flags=f, delays=[k % 3 for k in range(len(sizes))])
+    run_case(6, sizes, 0.05, 1, 0.9, steps=5, flags=f)
+    run_case(8, [300000], 0.25, 4, 0.9, steps=11, flags=f, same_init=False)
+    run_case(8, [6000, 77], 0.3, 2, 0.9, steps=8, flags=f, exchange="bf16")
+    run_case(8, [6000, 77], 0.3, 2, 0.9, steps=8, flags=f, exchange="fp8")          # general form
+    run_case(6, [6000, 77], 0.3, 2, 0.9, steps=8, flags=f, correction="eager")
+    run_case(8, [6000, 77], 0.3, 2, 0.9, steps=8, flags=f, optimizer="nadamw")       # NAdamW form
+    run_case(8, [6000, 77], 0.3, 4, 0.9, steps=12, flags=f, avg_interval=2)
+    o, g = run_case(8, [20000], 0.3, 2, 0.9, steps=6)                                # the default there
+    assert g.kernel_name() == "owner R=8 compact entries=128"
+    # consensus tracking is not available in two passes: the flag changes nothing, the value is still right
+    o, g = run_case(8, [20000], 0.3, 2, 0.9, steps=6, flags=binding.FLAG_TRACK_CONSENSUS)
+    assert g.kernel_name() == "owner R=8 compact entries=128"
+    assert abs(g.consensus_error(0) - o.consensus_error(0)) <= 1e-9 * o.consensus_error(0)
 
 
 def test_ragged_stage_sizes():
@@ -192,7 +214,7 @@ def test_averaging_interval(K, tau, p):
     run_case(4, [5000, 1024 * 2 + 3], p, tau, 0.9, steps=4 * K + tau + 1, avg_interval=K)
     run_case(3, [5000], p, tau, 0.9, steps=3 * K + tau + 1, avg_interval=K,
              flags=binding.FLAG_DIRECT_KERNEL)
-    run_case(8, [5000], p, tau, 0.9, steps=3 * K + tau + 1, avg_interval=K)   # pipelined kernel
+    run_case(8, [5000], p, tau, 0.9, steps=3 * K + tau + 1, avg_interval=K)   # eight replicas: whichever kernel is the default
 
 
 @pytest.mark.parametrize("tau,p", [(2, 0.05), (0, 0.3), (1, 1.0), (2, 0.4)])
@@ -538,7 +560,10 @@ def test_kernel_name_tells_which_kernel_runs():
     assert mk(8, 0.3, 0) == "owner R=8 sync" and mk(7, 0.05, 0) == "owner R=7 sync"
     assert mk(9, 0.3, 0) == "pipelined R=9 sync narrow"
     assert mk(8, 0.05, 2) == "pipelined R=8 compact wide"
-    assert mk(8, 0.3, 2) == "pipelined R=8 compact narrow"
+    assert mk(8, 0.3, 2) == "owner R=8 compact entries=128" and mk(6, 0.3, 2) == "owner R=6 compact entries=128"
+    assert mk(7, 0.3, 2) == "pipelined R=7 compact narrow"
+    assert mk(8, 0.3, 2, binding.FLAG_PIPELINED_KERNEL) == "pipelined R=8 compact narrow"
+    assert mk(8, 0.05, 2, binding.FLAG_OWNER_KERNEL) == "owner R=8 compact entries=32"
     assert mk(4, 0.05, 2, binding.FLAG_PIPELINED_KERNEL) == "pipelined R=4 compact wide"
     assert mk(4, 0.05, 2, binding.FLAG_DIRECT_KERNEL) == "direct R=4 compact"
     assert mk(4, 1.0, 2) == "direct R=4 dense"
