@@ -519,7 +519,8 @@ def test_coordinate_shards_equal_the_unsharded_stage(p, tau, flags):
 
 
 @pytest.mark.parametrize("R,p,tau,flags", [(3, 0.2, 1, 0), (4, 0.05, 2, 0), (8, 0.05, 2, 0), (8, 0.3, 0, 0),
-                                           (4, 0.3, 2, 2), (4, 1.0, 2, 0), (5, 0.4, 2, 4)])
+                                           (4, 0.3, 2, 2), (4, 1.0, 2, 0), (5, 0.4, 2, 4), (8, 0.3, 2, 0),
+                                           (6, 0.05, 1, 256), (4, 0.6, 2, 16 | 1024), (8, 1.0, 1, 64 | 1024)])
 def test_step_host_equals_step(R, p, tau, flags):
     # host gradients: copied stage by stage on the library's own stream, one launch per stage as
     # its gradients arrive -- the same state as the single launch on device gradients
