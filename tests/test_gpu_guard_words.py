@@ -146,6 +146,8 @@ def test_paths_for_more_selected_coordinates_than_the_fast_route_holds():
     run(4, [9000, 1024 * 3 + 5], 1.0, 2, flags=256)            # owner kernel: beyond the entries fetched ahead
     run(4, [9000, 1024 * 3 + 5], 0.05, 2, flags=1, expect_overflow=True)    # ring slot too small: dropped, reported
     run(8, [9000, 1024 * 3 + 5], 0.05, 2, flags=1, expect_overflow=True)
+    run(8, [9000, 1024 * 3 + 5], 0.05, 2, flags=1 | 256, expect_overflow=True)   # owner kernel in two passes
+    run(8, [9000, 1024 * 3 + 5], 1.0, 2, flags=256)                              # ... beyond the entries fetched ahead
     run(4, [9000], 0.3, 2, flags=128)                          # previous weights kept aside
 
 
