@@ -168,7 +168,8 @@ typedef struct asyncmesh_config {
  * (only where delta_j > 0), a copy of the previous weights (only with
  * ASYNCMESH_FLAG_KEEP_PREVIOUS) and the snapshot ring (compact: room for the
  * selected coordinates only, tau / K + 1 slots; dense, for large p: one position
- * per coordinate and replica, tau / K slots; K = avg_interval).  The library owns
+ * per coordinate and replica, tau / K slots, of 4-byte values, or of 2- or 1-byte
+ * values with ASYNCMESH_FLAG_RING_AS_EXCHANGED; K = avg_interval).  The library owns
  * all of it (obtained through cfg->alloc).
  * Moments, D and the ring start at zero, the step counter at 0, weights are
  * unset until asyncmesh_init_params.  The config and its arrays are copied.
