@@ -382,10 +382,16 @@ static int grid_for(uint64_t items, int threads)
 // kernel dispatch
 // ---------------------------------------------------------------------------
 
+// asyncmesh::pipelined for the owner kernel: 4 few, 7 some, 5 many entries fetched ahead; 6 synchronous
+static int owner_entries(int pipelined)
+{
+    return pipelined == 4 ? kOwnerEntriesFew : (pipelined == 7 ? kOwnerEntriesMid : kOwnerEntriesMany);
+}
+
 static KernelChoice pick_kernel(uint32_t R, int mode, int pipelined, bool general, uint32_t S)
 {
     if (pipelined >= 4) {
-        const int entries = pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany;
+        const int entries = owner_entries(pipelined);
         return general ? pick_owner_general(R, mode, entries, S) : pick_owner_common(R, mode, entries, S);
     }
     if (pipelined && R <= 8)
@@ -563,7 +569,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
 
     // the compact ring has two kernels; which one is fixed for the handle's life
     h->pipelined = 0;   // 0 direct, 1 pipelined wide, 2 pipelined narrow, 3 pipelined narrow synchronous,
-                        // 4 to 6 owner (below)
+                        // 4 to 7 owner (below)
     // synchronous mode: the stash route pays while most float4 groups are only partly
     // selected; towards p = 1 the direct kernel writes whole groups and wins
     if (h->mode == kSync && !(cfg->flags & ASYNCMESH_FLAG_DIRECT_KERNEL) &&
@@ -576,7 +582,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     }
 
     // Up to four replicas: the owner kernel (4: few ring / d entries fetched ahead per
-    // group, 5: many, 6: synchronous) wherever one of the two pipelined shapes would run,
+    // group, 7: some, 5: many, 6: synchronous) wherever one of the two pipelined shapes would run,
     // unless a flag asks for another kernel.  1B layout, tau = 4, ms per step, pipelined
     // against owner: p = 0.01 21.6 / 20.7, 0.05 23.4 / 22.7, 0.1 26.2 / 23.9, 0.25 30.9 / 25.6,
     // 0.5 37.4 / 29.0; tau = 0: 20.8 to 24.4 / 20.5 to 20.7 at every p.
@@ -608,7 +614,7 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     const bool few_entries = group_mean + 4.0 * std::sqrt(group_mean * (1.0 - cfg->p)) <= (double)kOwnerEntriesFew;
     if ((R <= 4 || (R <= 8 && h->mode == kSync) || two_pass) && !is_dense(h->mode) &&
         (owner_asked || (owner_default && (!two_pass || !few_entries))))
-        h->pipelined = h->mode == kSync ? 6 : (few_entries ? 4 : 5);
+        h->pipelined = h->mode == kSync ? 6 : few_entries ? 4 : (!two_pass && group_mean <= 96.0) ? 7 : 5;
 
 
     auto bail = [&](int code, const char *what) {
@@ -687,12 +693,12 @@ extern "C" int asyncmesh_create(const asyncmesh_config *cfg, asyncmesh **out)
     h->nadam_form = h->pipelined >= 4 && nadam_only;
     h->general = general && !h->nadam_form;
     h->kernel = h->nadam_form
-        ? pick_owner_nadamw(R, h->mode, h->pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany, S)
+        ? pick_owner_nadamw(R, h->mode, owner_entries(h->pipelined), S)
         : pick_kernel(R, h->mode, h->pipelined, general, S);
     if ((cfg->flags & ASYNCMESH_FLAG_TRACK_CONSENSUS) && h->pipelined >= 4 && !general &&
         (R <= 4 || h->mode == kSync)) {
         h->tracking = true;
-        h->kernel = pick_owner_tracking(R, h->mode, h->pipelined == 4 ? kOwnerEntriesFew : kOwnerEntriesMany, S);
+        h->kernel = pick_owner_tracking(R, h->mode, owner_entries(h->pipelined), S);
     }
     int sms = 0, per_sm = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
@@ -1171,6 +1177,7 @@ extern "C" int asyncmesh_kernel_name(const asyncmesh *h, char *buf, size_t cap)
     case 2: case 3: snprintf(buf, cap, "pipelined R=%u %s narrow%s", h->R, mode, form); break;
     case 4: snprintf(buf, cap, "owner R=%u %s entries=%d%s", h->R, mode, kOwnerEntriesFew, form); break;
     case 5: snprintf(buf, cap, "owner R=%u %s entries=%d%s", h->R, mode, kOwnerEntriesMany, form); break;
+    case 7: snprintf(buf, cap, "owner R=%u %s entries=%d%s", h->R, mode, kOwnerEntriesMid, form); break;
     default: snprintf(buf, cap, "owner R=%u %s%s", h->R, mode, form);
     }
     return ASYNCMESH_OK;

@@ -29,7 +29,7 @@ KernelChoice pick_pipelined_few_general(uint32_t R, int shape, uint32_t S);
 KernelChoice pick_pipelined_many_common(uint32_t R, int shape, uint32_t S);    // R = 9..16
 KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S);
 // Owner kernel (R = 1..4; R = 5..8 for kSync; R = 6 and 8 for kCompact as two passes over each group).  mode: kCompact or kSync; entries: ring / d entries per group
-// of 256 coordinates fetched ahead (kOwnerEntriesFew or kOwnerEntriesMany).
+// of 256 coordinates fetched ahead (kOwnerEntriesFew, kOwnerEntriesMid or kOwnerEntriesMany).
 // Shape, measured on the 1B layout (R = 4, p = 0.05, ms per step): one replica row per
 // unit and 8 coordinates per lane (1 KB contiguous per array row and request) 22.7;
 // two rows per unit 23.0; 4 coordinates per lane (512-byte requests) 24.3 to 24.8 whatever
@@ -40,7 +40,12 @@ KernelChoice pick_pipelined_many_general(uint32_t R, int shape, uint32_t S);
 // copies are tracked apart from the dense ones).
 constexpr int owner_stages(int mode) { return mode == kSync ? 2 : 3; }
 constexpr int kOwnerV = 2;
-constexpr int kOwnerEntriesFew = 32, kOwnerEntriesMany = 128;
+// Entries fetched ahead per group: 32 keep three blocks per SM with room to spare; 64 still fit three blocks
+// (72 KB each) and serve the medium subsets, where half of the groups then read some entries in place; 128 take
+// the kernel down to two blocks per SM.  1B layout, tau = 4, ms per step with 64 against 128: p = 0.1 23.85 /
+// 24.33, 0.15 24.66 / 25.61, 0.25 26.33 / 26.62, 0.5 30.43 / 30.31 (96: 25.1, 25.8, 26.7, 33.9).  In two passes
+// (six and eight replicas) 64 lose to 128 (350M layout, p = 0.25: 19.3 / 18.8), so that form knows two sizes.
+constexpr int kOwnerEntriesFew = 32, kOwnerEntriesMid = 64, kOwnerEntriesMany = 128;
 // replica rows per unit: one up to four replicas; with more, two where that divides R (8 KB units)
 constexpr int owner_ru(int R) { return (R > 4 && R % 2 == 0) ? 2 : 1; }
 KernelChoice pick_owner_common(uint32_t R, int mode, int entries, uint32_t S);

@@ -147,8 +147,9 @@ template <int R>
 static KernelChoice owner(int mode, int entries, uint32_t S)
 {
     if (mode == kSync) return owner_as<R, 1, kSync>(S);
-    return entries == kOwnerEntriesFew ? owner_as<R, kOwnerEntriesFew, kCompact>(S)
-                                       : owner_as<R, kOwnerEntriesMany, kCompact>(S);
+    return entries == kOwnerEntriesFew   ? owner_as<R, kOwnerEntriesFew, kCompact>(S)
+           : entries == kOwnerEntriesMid ? owner_as<R, kOwnerEntriesMid, kCompact>(S)
+                                         : owner_as<R, kOwnerEntriesMany, kCompact>(S);
 }
 
 #if AM_PART == 7

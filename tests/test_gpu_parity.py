@@ -556,7 +556,8 @@ def test_kernel_name_tells_which_kernel_runs():
     mk = lambda R, p, tau, flags=0, **kw: am().AsyncMesh(R, [5000], p=p, tau=tau, ema_beta=0.9, flags=flags,
                                                           **dict(HP, **kw)).kernel_name()
     assert mk(4, 0.05, 2) == "owner R=4 compact entries=32"
-    assert mk(4, 0.3, 2) == "owner R=4 compact entries=128"
+    assert mk(4, 0.3, 2) == "owner R=4 compact entries=64" and mk(4, 0.1, 2) == "owner R=4 compact entries=64"
+    assert mk(4, 0.4, 4) == "owner R=4 compact entries=128" and mk(3, 0.36, 2) == "owner R=3 compact entries=64"
     assert mk(3, 0.3, 0) == "owner R=3 sync"
     assert mk(8, 0.3, 0) == "owner R=8 sync" and mk(7, 0.05, 0) == "owner R=7 sync"
     assert mk(9, 0.3, 0) == "pipelined R=9 sync narrow"
@@ -570,7 +571,7 @@ def test_kernel_name_tells_which_kernel_runs():
     assert mk(4, 1.0, 2) == "direct R=4 dense"
     assert mk(4, 1.0, 0) == "direct R=4 sync"
     assert mk(4, 0.05, 2, optimizer="nadamw") == "owner R=4 compact entries=32 nadamw"
-    assert mk(4, 0.3, 2, optimizer="nadamw") == "owner R=4 compact entries=128 nadamw"
+    assert mk(4, 0.3, 2, optimizer="nadamw") == "owner R=4 compact entries=64 nadamw"
     assert mk(4, 0.05, 0, optimizer="nadamw") == "owner R=4 sync nadamw"
     assert mk(8, 0.05, 0, optimizer="nadamw") == "owner R=8 sync nadamw"
     assert mk(4, 0.3, 0, binding.FLAG_FP8_EXCHANGE) == "owner R=4 sync general"
