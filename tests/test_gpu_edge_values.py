@@ -148,3 +148,20 @@ def test_edge_values_nadamw():
     run(4, 2 * 1024 + 7, 0.3, 2, flags_of("pipelined"), optimizer="nadamw")      # pipelined kernel, general form
     run(4, 2 * 1024 + 7, 0.3, 0, 0, optimizer="nadamw", steps=4)
     run(8, 2 * 1024 + 7, 0.3, 2, 0, optimizer="nadamw")
+
+
+@pytest.mark.parametrize("case", range(48))
+def test_edge_values_random_configuration(case):
+    # the hand-built special values through whatever kernel, form and ring mode a seeded draw selects
+    rng = np.random.default_rng(0xED6E + case)
+    R = int(rng.choice([1, 2, 3, 4, 4, 5, 6, 8, 8, 12]))
+    n = int(rng.choice([1024 + 7, 2 * 1024 + 41, 3 * 1024 + 5]))
+    p = float(rng.choice([0.05, 0.2, 0.5, 1.0]))
+    tau = int(rng.choice([0, 1, 2, 3]))
+    exchange = str(rng.choice(["fp32", "fp32", "bf16", "fp8"]))
+    snapshot = "as-exchanged" if exchange != "fp32" and tau > 0 and rng.random() < 0.4 else "own-fp32"
+    kernel = str(rng.choice(["default", "default", "direct", "pipelined", "owner"]))
+    flags = 0 if snapshot == "as-exchanged" else flags_of(kernel)
+    optimizer = str(rng.choice(["adamw", "adamw", "nadamw"]))
+    run(R, n, p, tau, flags, exchange=exchange, steps=int(rng.integers(4, 8)), seed=case, optimizer=optimizer,
+        snapshot=snapshot)
